@@ -1,0 +1,435 @@
+#!/usr/bin/env python
+"""Benchmark of the A2SGD per-worker gradient path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
+
+One "step" is one whole pass of the hot path — encode (two local means per worker), average of
+the 2P scalars, decode + residual update + SGD step — over all P simulated workers of the
+workload.  Prints ONE JSON line (rank 0).
+
+* ``value``      model parameters per second (n / step time), inputs resident in HBM.
+* ``e2e``        the same metric through ``a2sgd_step_host``: every step copies that step's
+                 gradients from pinned host memory and reads the 2P+2 means back.
+* ``roofline``   the decode/update kernel (the larger of the two launches of a step) timed
+                 alone with CUDA events: algorithmic bytes / duration against the measured
+                 copy bandwidth of this machine.
+* ``cpu_baseline`` the CPU oracle, as it stands, on a bounded sample of the same workload.
+
+With N > 1 (under torchrun) every rank runs an independent replica of the workload on its own
+GPU — the benchmarked path has no exchange between GPUs — and the time is the max over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "a2sgd_step_model_params_per_s"
+UNIT = "params/s"
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+
+# DRAM bytes (read + write) per model element of the decode/update kernel, from the ncu
+# captures summarised under profiles/ (None until a capture exists for that P).
+NCU_DECODE_TRAFFIC_PER_ELEMENT = {}
+
+
+def algorithmic_bytes_per_model_element(P: int, shared_w: bool = True) -> dict:
+    """EF mode, fp32: K1 reads g and e of every worker; K3 reads g, e, w and writes e, w."""
+    encode = 8 * P
+    decode = (12 * P + 8) if shared_w else 20 * P
+    return {"encode": encode, "decode": decode, "step": encode + decode}
+
+
+def measured_peak_gbs():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback (no MEASURED_PEAKS.json)"
+
+
+# ----------------------------------------------------------------------------- clocks
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, device_index: int):
+        import torch
+        self.proc = None
+        self.path = None
+        try:
+            uuid = str(torch.cuda.get_device_properties(device_index).uuid)
+            ident = uuid if uuid.startswith("GPU-") else "GPU-" + uuid
+        except Exception:
+            ident = str(device_index)
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.out = open(self.path, "w")
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", ident, f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=self.out, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.out.close()
+        sm, smax, power, reasons = [], [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        with open(self.path) as f:
+            for line in f:
+                parts = [p.strip() for p in line.split(",")]
+                if len(parts) < 7:
+                    continue
+                try:
+                    sm.append(float(parts[0]))
+                    smax.append(float(parts[1]))
+                    power.append(float(parts[2]))
+                except ValueError:
+                    continue
+                for name, val in zip(names, parts[3:7]):
+                    if val.lower().startswith("active"):
+                        reasons.add(name)
+        os.unlink(self.path)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        sm.sort()
+        return {"sm_mhz": sm[len(sm) // 2], "sm_max_mhz": max(smax), "power_w_max": max(power),
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ----------------------------------------------------------------------------- reference arm
+def oracle_sample_rate(wl, target_seconds: float, gen_device="cpu"):
+    """Times the CPU oracle (single thread, unmodified) on a prefix sample of the workload's
+    flat vector: all P workers, the first n_s elements of each.  Returns a dict."""
+    import numpy as np
+    import torch
+    import oracle
+    from paper_2006_07405_b200 import workloads as W
+
+    def run(n_s, steps=1):
+        g = torch.empty((wl.P, n_s))
+        sub = W.scaled(wl, max(1, wl.n // n_s))
+        gfull = torch.empty((wl.P, sub.n))
+        W.fill_gradients(sub, 0, gfull)
+        reps = (n_s + sub.n - 1) // sub.n
+        g.copy_(gfull.repeat(1, reps)[:, :n_s])
+        g = g.numpy()
+        e = np.zeros_like(g)
+        w = np.zeros(n_s, np.float32)
+        t0 = time.perf_counter()
+        for _ in range(steps):
+            oracle.step(w, g, e, wl.lr, mode=oracle.MODE_EF)
+        return (time.perf_counter() - t0) / steps
+
+    probe_n = min(wl.n, 1 << 20)
+    t_probe = run(probe_n)
+    n_s = int(min(wl.n, max(probe_n, probe_n * target_seconds / max(t_probe, 1e-9))))
+    t = run(n_s)
+    return {"value": n_s / t, "unit": UNIT, "cores": 1, "kind": "oracle",
+            "sample": f"first {n_s} of {wl.n} elements of each of the {wl.P} workers, 1 step, {t:.2f} s",
+            "_n_s": n_s, "_seconds": t}
+
+
+def run_reference(args):
+    """bench.py --impl reference: the oracle on the host cores, rank 0 only."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from paper_2006_07405_b200 import workloads as W
+    wl = W.get_workload(args.workload)
+    per_step_budget = max(0.5, min(10.0, 120.0 / max(1, args.steps + args.warmup)))
+    first = oracle_sample_rate(wl, per_step_budget)
+    n_s = first["_n_s"]
+    import numpy as np
+    import torch
+    import oracle
+    sub = W.scaled(wl, max(1, wl.n // n_s))
+    gfull = torch.empty((wl.P, sub.n))
+    W.fill_gradients(sub, 0, gfull)
+    g = gfull.repeat(1, (n_s + sub.n - 1) // sub.n)[:, :n_s].contiguous().numpy()
+    e = np.zeros_like(g)
+    w = np.zeros(n_s, np.float32)
+    for _ in range(args.warmup):
+        oracle.step(w, g, e, wl.lr, mode=oracle.MODE_EF)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle.step(w, g, e, wl.lr, mode=oracle.MODE_EF)
+    t = (time.perf_counter() - t0) / max(1, args.steps)
+    value = n_s / t
+    sample = f"first {n_s} of {wl.n} elements of each of the {wl.P} workers per step"
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": t * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": dict(W.describe(wl), note="CPU oracle, single thread, bounded sample"),
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line), flush=True)
+
+
+# ----------------------------------------------------------------------------- device arm
+def time_workload(wl, steps, warmup, dev, *, with_roofline=True, with_e2e=True, dist=None):
+    """Runs the timed regions for one workload on this rank's GPU.  Returns a dict of results."""
+    import torch
+    from paper_2006_07405_b200 import binding as B
+    from paper_2006_07405_b200 import workloads as W
+
+    n, P = wl.n, wl.P
+    torch.cuda.set_device(dev)
+    g = torch.empty((P, n), device=dev)
+    e = torch.zeros((P, n), device=dev)
+    w = torch.empty(n, device=dev)
+    W.fill_gradients(wl, 0, g)
+    W.init_weights(wl, w)
+    ctx = B.a2sgd_create(n, P, dev.index, B.MODE_EF)
+    info = B.a2sgd_launch_info(ctx, shared_w=True)
+    launches_per_step = 1 if info["single_launch"] else 2
+
+    def barrier():
+        torch.cuda.synchronize(dev)
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize(dev)
+
+    for _ in range(max(warmup, 3)):
+        B.a2sgd_step(ctx, w, g, e, wl.lr)
+    barrier()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    wall0 = time.time()
+    ev0.record()
+    for _ in range(steps):
+        B.a2sgd_step(ctx, w, g, e, wl.lr)
+    ev1.record()
+    barrier()
+    wall1 = time.time()
+    ms = ev0.elapsed_time(ev1)
+    if dist is not None:
+        t = torch.tensor([ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    res = {"ms_total": ms, "ms_per_step": ms / steps, "launches": launches_per_step * steps,
+           "launch_info": info, "wall": (wall0, wall1)}
+    *_, status = B.a2sgd_read_stats(ctx)
+    res["device_status"] = status
+
+    if with_roofline:
+        # the decode/update kernel alone, same launch configuration as inside a2sgd_step
+        lm = torch.zeros((P, 2), device=dev)
+        gm = torch.zeros(2, device=dev)
+        k_steps = max(5, min(steps, 200))
+        enc_ms = dec_ms = 0.0
+        evs = [torch.cuda.Event(enable_timing=True) for _ in range(3 * k_steps)]
+        for i in range(k_steps):
+            evs[3 * i].record()
+            B.a2sgd_encode(ctx, g, e, lm)
+            B.a2sgd_global_average(ctx, lm, gm)
+            evs[3 * i + 1].record()
+            B.a2sgd_decode_update(ctx, w, g, e, lm, gm, wl.lr)
+            evs[3 * i + 2].record()
+        torch.cuda.synchronize(dev)
+        for i in range(k_steps):
+            enc_ms += evs[3 * i].elapsed_time(evs[3 * i + 1])
+            dec_ms += evs[3 * i + 1].elapsed_time(evs[3 * i + 2])
+        res["encode_ms"] = enc_ms / k_steps
+        res["decode_ms"] = dec_ms / k_steps
+
+    if with_e2e:
+        try:
+            g_host = torch.empty((P, n)).pin_memory()
+        except Exception:
+            g_host = torch.empty((P, n))
+        g_host.copy_(g)
+        means = torch.zeros(2 * P + 2).pin_memory()
+        e2e_steps = max(2, min(steps, 10))
+        for _ in range(2):
+            B.a2sgd_step_host(ctx, w, g_host, g, e, wl.lr, means)
+        barrier()
+        ev0.record()
+        for _ in range(e2e_steps):
+            B.a2sgd_step_host(ctx, w, g_host, g, e, wl.lr, means)
+        ev1.record()
+        barrier()
+        ms2 = ev0.elapsed_time(ev1)
+        if dist is not None:
+            t = torch.tensor([ms2], device=dev, dtype=torch.float64)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms2 = float(t.item())
+        res["e2e_ms_per_step"] = ms2 / e2e_steps
+        res["e2e_steps"] = e2e_steps
+        res["h2d_bytes"] = P * n * 4
+        res["d2h_bytes"] = (2 * P + 2) * 4
+        del g_host
+    ctx.destroy()
+    del g, e, w
+    torch.cuda.empty_cache()
+    return res
+
+
+def load_loop_for_clocks(wl, dev, seconds):
+    """Keeps the same kernels running so the clock sampler sees the GPU under this load."""
+    import torch
+    from paper_2006_07405_b200 import binding as B
+    from paper_2006_07405_b200 import workloads as W
+    n, P = wl.n, wl.P
+    g = torch.empty((P, n), device=dev)
+    e = torch.zeros((P, n), device=dev)
+    w = torch.zeros(n, device=dev)
+    W.fill_gradients(wl, 0, g)
+    ctx = B.a2sgd_create(n, P, dev.index, B.MODE_EF)
+    t0 = time.time()
+    while time.time() - t0 < seconds:
+        for _ in range(50):
+            B.a2sgd_step(ctx, w, g, e, wl.lr)
+        torch.cuda.synchronize(dev)
+    ctx.destroy()
+
+
+def summarise(wl, res, n_gpus, peak_gbs):
+    b = algorithmic_bytes_per_model_element(wl.P)
+    t = res["ms_per_step"] * 1e-3
+    out = {"n": wl.n, "P": wl.P, "ms_per_step": res["ms_per_step"],
+           "model_params_per_s": n_gpus * wl.n / t, "worker_params_per_s": n_gpus * wl.n * wl.P / t,
+           "step_GBps": b["step"] * wl.n / t / 1e9,
+           "step_frac_of_8TBps": b["step"] * wl.n / t / 1e9 / NOMINAL_HBM_GBS,
+           "step_frac_of_measured_peak": b["step"] * wl.n / t / 1e9 / peak_gbs}
+    if "decode_ms" in res:
+        out["encode_ms"] = res["encode_ms"]
+        out["decode_ms"] = res["decode_ms"]
+        out["encode_GBps"] = b["encode"] * wl.n / (res["encode_ms"] * 1e-3) / 1e9
+        out["decode_GBps"] = b["decode"] * wl.n / (res["decode_ms"] * 1e-3) / 1e9
+    return out
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--workload", default="c2_lstm_ptb")
+    ap.add_argument("--impl", default="native", choices=["native", "reference"])
+    ap.add_argument("--no-extra", action="store_true", help="skip the extra c4/c5 measurements at N=1")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+
+    if args.impl == "reference":
+        run_reference(args)
+        return
+
+    import torch
+    from paper_2006_07405_b200 import binding as B
+    from paper_2006_07405_b200 import workloads as W
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the A2SGD path has no CPU fallback")
+    B.lib()  # fail loudly if the CUDA library has not been built
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist_mod.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+        dist = dist_mod
+    n_gpus = world
+    dev = torch.device("cuda", local_rank)
+    torch.cuda.set_device(dev)
+    wl = W.get_workload(args.workload)
+    peak_gbs, peak_src = measured_peak_gbs()
+    steps, warmup = max(1, args.steps), max(3, args.warmup)
+
+    sampler = ClockSampler(local_rank) if rank == 0 else None
+    res = time_workload(wl, steps, warmup, dev, dist=dist)
+    if rank == 0 and res["ms_total"] < 1500.0:
+        load_loop_for_clocks(wl, dev, 1.5)
+    clocks = sampler.stop() if sampler else None
+    if clocks is not None:
+        clocks["sampled_over"] = "timed region" if res["ms_total"] >= 1500.0 else \
+            "timed region plus 1.5 s of the same step loop (timed region shorter than the sampling period allows)"
+
+    extra = {}
+    if rank == 0 and world == 1 and not args.no_extra and args.workload == "c2_lstm_ptb":
+        free_b, _ = torch.cuda.mem_get_info(dev)
+        for name in ("c1_flat_1m", "c3_resnet50", "c4_vgg16", "c5_gpt2_xl"):
+            w2 = W.get_workload(name)
+            need = (2 * w2.P + 1) * w2.n * 4 * 1.05
+            if need > free_b:
+                extra[name] = {"skipped": "not enough free device memory"}
+                continue
+            k = 20 if w2.n > 10 ** 9 else (100 if w2.n > 10 ** 7 else 1000)
+            r2 = time_workload(w2, k, 3, dev, with_e2e=False)
+            extra[name] = summarise(w2, r2, 1, peak_gbs)
+
+    if dist is not None:
+        dist.barrier()
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    b = algorithmic_bytes_per_model_element(wl.P)
+    t = res["ms_per_step"] * 1e-3
+    value = n_gpus * wl.n / t
+    dec_t = res["decode_ms"] * 1e-3
+    achieved = b["decode"] * wl.n / dec_t / 1e9
+    traffic_per_el = NCU_DECODE_TRAFFIC_PER_ELEMENT.get(wl.P)
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": n_gpus, "steps": steps, "warmup": warmup,
+        "ms_per_step": res["ms_per_step"], "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32", "data": "synthetic",
+        "config": dict(W.describe(wl), mode="EF", w_layout="one shared w", resident_GB=(2 * wl.P + 1) * wl.n * 4 / 1e9,
+                       l2="inputs larger than L2: every step streams the whole resident set",
+                       parallelism=f"{n_gpus} independent replica(s), no collective",
+                       worker_params_per_s=n_gpus * wl.n * wl.P / t,
+                       step_GBps=b["step"] * wl.n / t / 1e9,
+                       step_frac_of_8TBps=b["step"] * wl.n / t / 1e9 / NOMINAL_HBM_GBS,
+                       step_frac_of_measured_peak=b["step"] * wl.n / t / 1e9 / peak_gbs,
+                       bytes_per_model_element=b, launch=res["launch_info"],
+                       encode_ms=res["encode_ms"], decode_ms=res["decode_ms"],
+                       device_status=res["device_status"]),
+        "gpu_launches": res["launches"],
+        "clocks": clocks,
+        "e2e": {"value": n_gpus * wl.n / (res["e2e_ms_per_step"] * 1e-3), "unit": UNIT,
+                "h2d_bytes_per_step": res["h2d_bytes"], "d2h_bytes_per_step": res["d2h_bytes"],
+                "ms_per_step": res["e2e_ms_per_step"], "steps": res["e2e_steps"],
+                "api": "a2sgd_step_host (pinned host gradients in, 2P+2 means out)"},
+        "roofline": {"bound": "hbm", "kernel": "decode/update (K3)", "achieved": achieved, "peak": peak_gbs,
+                     "unit": "GB/s", "frac": achieved / peak_gbs, "peak_source": peak_src,
+                     "traffic": traffic_per_el * wl.n if traffic_per_el else None,
+                     "algorithmic_bytes": b["decode"] * wl.n, "launch_ms": res["decode_ms"],
+                     "encode_kernel": {"achieved": b["encode"] * wl.n / (res["encode_ms"] * 1e-3) / 1e9,
+                                       "frac": b["encode"] * wl.n / (res["encode_ms"] * 1e-3) / 1e9 / peak_gbs,
+                                       "launch_ms": res["encode_ms"],
+                                       "note": "encode + stand-alone global-average launch"}},
+    }
+    if extra:
+        line["other_workloads"] = extra
+    if not args.no_cpu_baseline and world == 1:
+        cb = oracle_sample_rate(wl, 10.0)
+        line["cpu_baseline"] = {k: v for k, v in cb.items() if not k.startswith("_")}
+    print(json.dumps(line), flush=True)
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

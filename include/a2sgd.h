@@ -1,0 +1,159 @@
+/*
+ * liba2sgd — the per-worker gradient path of A2SGD (two-level gradient
+ * averaging) as CUDA kernels for sm_100a behind a plain C ABI.
+ *
+ * What the path computes (Section 3.1, Eq. 2 and Algorithm 1 of the paper).
+ * For every one of P data-parallel workers holding an n-element fp32 vector v:
+ *   pos(v)_i = 1 if v_i >= 0 else 0,  neg(v) = 1 - pos(v)
+ *   mu_pos(v) = mean of the entries v_i >= 0      (0 for an empty group)
+ *   mu_neg(v) = mean of |v_i| over entries v_i < 0 (0 for an empty group)
+ * The P pairs (mu_pos, mu_neg) — 64 bits per worker — are averaged, unweighted,
+ * into the global pair (m_pos, m_neg) (Algorithm 1 line 5).  Each worker then
+ * rebuilds a dense gradient from the two global means, updates its local
+ * error vector and applies w <- w - lr * g_hat (Algorithm 1 lines 4, 6, 7).
+ *
+ * Two modes, chosen at a2sgd_create:
+ *   A2SGD_MODE_EF    error feedback carried between iterations:
+ *                    v = g + e,  g_hat = pos(v)*m_pos - neg(v)*m_neg,
+ *                    e <- v - g_hat        (so e_new + g_hat == g + e_old).
+ *   A2SGD_MODE_ALG1  Algorithm 1 as printed (same-iteration add-back, Eq. 13):
+ *                    v = g,  eps = g - (pos*mu_pos^p - neg*mu_neg^p),
+ *                    g_hat = eps + pos*m_pos - neg*m_neg; eps is stored to
+ *                    `err` only when the caller passes a non-NULL err.
+ *
+ * The P workers are simulated as P buffers on one GPU: worker p's vector is
+ * at `base + p*stride` (stride in ELEMENTS, 64-bit).  Weights are either one
+ * replica per worker (w_stride >= n, the layout of Algorithm 1) or one shared
+ * vector (w_stride == 0), which receives the worker-mean of the reconstructed
+ * gradients, w <- w - (lr/P) * sum_p g_hat^p — the mean of the P replicas.
+ *
+ * Pointers.  Unless an argument is marked HOST it is DEVICE memory on the
+ * context's device, owned by the caller, at least 4-byte aligned.  The
+ * library never allocates, frees or retains these buffers.  Any alignment
+ * that is a multiple of 4 bytes is computed correctly; the fast kernels
+ * need 16-byte aligned bases and strides that are multiples of 4 elements.
+ * `grad` is never written.
+ *
+ * Execution.  Every call enqueues its kernels on `stream` (a cudaStream_t
+ * passed as void*, NULL = default stream) and returns without waiting, except
+ * a2sgd_read_stats and a2sgd_step_host, which synchronise `stream`.
+ * Conditions seen by the host (bad arguments) return a negative status and
+ * launch nothing.  Conditions seen on the device (non-finite sums, a bounded
+ * wait that ran out) are latched in a status word read by a2sgd_read_stats.
+ * Results are bitwise reproducible for a fixed (n, P, strides' alignment,
+ * device, build): no floating-point atomics, fixed-order combines.
+ * A context owns only small scratch (per-CTA partial sums, 2P+2 means, P
+ * counts, tickets, status); use one context per stream; a context is not
+ * thread-safe.  Limits: 1 <= n < 2^40, 1 <= P <= 1024.
+ */
+#ifndef A2SGD_H_
+#define A2SGD_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct a2sgd_ctx a2sgd_ctx;
+
+enum a2sgd_status {
+    A2SGD_OK = 0,
+    A2SGD_ERR_ARG = -1,       /* NULL pointer, n or P out of range, stride < n, bad flag */
+    A2SGD_ERR_ALIGN = -2,     /* a float pointer that is not 4-byte aligned */
+    A2SGD_ERR_CUDA = -3,      /* a CUDA runtime call failed */
+    A2SGD_ERR_TIMEOUT = -4,   /* a bounded device-side wait ran out (latched in the status word) */
+    A2SGD_ERR_NONFINITE = -5, /* a group sum was NaN or Inf (latched in the status word) */
+    A2SGD_ERR_NOMEM = -6,     /* scratch allocation failed */
+    A2SGD_ERR_TOO_LARGE = -7  /* n*P exceeds what the single-launch path can hold on chip */
+};
+
+enum a2sgd_flags {
+    A2SGD_MODE_EF = 0,                /* default */
+    A2SGD_MODE_ALG1 = 1,
+    A2SGD_FORCE_TWO_PASS = 1 << 4,    /* a2sgd_step never takes the single-launch path */
+    A2SGD_FORCE_COOPERATIVE = 1 << 5  /* a2sgd_step always takes it; A2SGD_ERR_TOO_LARGE if it cannot */
+};
+
+/* Creates a context for vectors of n elements and P workers on `device`
+ * (made current for the duration of each call, then restored).  Allocates
+ * the scratch listed above with cudaMalloc.  *out is NULL on failure. */
+int a2sgd_create(a2sgd_ctx **out, uint64_t n, uint32_t P, int device, uint32_t flags);
+
+/* Frees the scratch.  NULL is accepted. */
+int a2sgd_destroy(a2sgd_ctx *ctx);
+
+/* Algorithm 1 line 3 (Section 3.1): the two local means of every worker.
+ *   grad        [P] vectors of n floats, worker stride grad_stride (>= n)
+ *   err         EF: the retained error, same layout (required).  ALG1: ignored, may be NULL
+ *   local_means out, [P][2] floats = {mu_pos, mu_neg}: exactly 8 bytes per worker
+ *   pos_counts  out, [P] uint64 = #{i : v_i >= 0}, may be NULL
+ *   pos_mask    out, [P][ceil(n/32)] uint32, bit b of word j = pos of element 32*j+b,
+ *               unused high bits of the last word 0; may be NULL */
+int a2sgd_encode(a2sgd_ctx *ctx, const float *grad, int64_t grad_stride,
+                 const float *err, int64_t err_stride, float *local_means,
+                 uint64_t *pos_counts, uint32_t *pos_mask, void *stream);
+
+/* Algorithm 1 line 5, with the P workers on one device: the unweighted mean
+ * of the P pairs, summed in worker order in fp64, rounded once to fp32.
+ *   local_means  in,  [P][2]      global_means  out, [2] = {m_pos, m_neg} */
+int a2sgd_global_average(a2sgd_ctx *ctx, const float *local_means,
+                         float *global_means, void *stream);
+
+/* Algorithm 1 lines 4, 6 and 7 fused: reconstruct, update the residual,
+ * apply the SGD step.  Reads grad, err (EF) and w once, writes err and w once.
+ *   w            in/out; w_stride == 0: one shared vector, else >= n: one per worker
+ *   err          EF: in/out (required).  ALG1: out (eps), may be NULL
+ *   local_means  in, [P][2]; read in ALG1 mode only (may be NULL in EF)
+ *   global_means in, [2]
+ *   lr           learning rate of this step */
+int a2sgd_decode_update(a2sgd_ctx *ctx, float *w, int64_t w_stride,
+                        const float *grad, int64_t grad_stride,
+                        float *err, int64_t err_stride,
+                        const float *local_means, const float *global_means,
+                        float lr, void *stream);
+
+/* One whole loop body of Algorithm 1 (lines 3-7) for all P workers: encode,
+ * average the 2P scalars, decode/update.  The means stay in the context and
+ * can be read back with a2sgd_read_stats.  Two launches for large n; a
+ * single cooperative launch that keeps v on chip when n*P is small enough
+ * (see a2sgd_flags). */
+int a2sgd_step(a2sgd_ctx *ctx, float *w, int64_t w_stride,
+               const float *grad, int64_t grad_stride,
+               float *err, int64_t err_stride, float lr, void *stream);
+
+/* a2sgd_step for a caller whose fresh gradients sit in HOST memory (pinned
+ * memory makes the copies asynchronous): copies grad_host -> grad_staging
+ * worker by worker, runs the step, copies the 2P local and 2 global means
+ * to means_host and synchronises `stream`.
+ *   grad_host     HOST, [P] vectors of n floats, stride grad_host_stride
+ *   grad_staging  device, caller-owned, [P] vectors with stride grad_stride
+ *   means_host    HOST, out, [2P + 2] floats: local pairs then the global pair */
+int a2sgd_step_host(a2sgd_ctx *ctx, float *w, int64_t w_stride,
+                    const float *grad_host, int64_t grad_host_stride,
+                    float *grad_staging, int64_t grad_stride,
+                    float *err, int64_t err_stride, float lr,
+                    float *means_host, void *stream);
+
+/* Synchronises `stream`, then copies the context's latest means and counts
+ * (written by a2sgd_step / a2sgd_encode) to HOST memory and returns the
+ * latched device status (A2SGD_OK, A2SGD_ERR_TIMEOUT or A2SGD_ERR_NONFINITE)
+ * in *device_status, clearing the latch.  Any out pointer may be NULL.
+ *   local_means_host [P][2], global_means_host [2], pos_counts_host [P] */
+int a2sgd_read_stats(a2sgd_ctx *ctx, float *local_means_host,
+                     float *global_means_host, uint64_t *pos_counts_host,
+                     int *device_status, void *stream);
+
+/* Launch geometry of the context's kernels, for benchmarks and reports:
+ * out[0] = CTAs of the encode launch, out[1] = CTAs of the decode launch,
+ * out[2] = threads per CTA, out[3] = 1 if a2sgd_step takes the single-launch
+ * path for this (n, P), out[4] = SM count.  HOST pointer. */
+int a2sgd_launch_info(a2sgd_ctx *ctx, int64_t w_stride, uint32_t out[5]);
+
+/* Static, never NULL. */
+const char *a2sgd_status_string(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* A2SGD_H_ */

@@ -1,0 +1,209 @@
+"""Thin ctypes binding of liba2sgd (the C ABI declared in include/a2sgd.h).
+
+Argument marshalling only: every step of the path runs in the library's CUDA
+kernels.  Tensors are used for device memory and streams, nothing else.  There
+is no fallback: if the shared library has not been built, or a call returns a
+negative status, an exception is raised.
+
+Layout conventions (same as the header): ``grad`` / ``err`` are float32 CUDA
+tensors ``[P, >= n]`` with unit inner stride (row p = worker p); ``w`` is
+``[>= n]`` (one shared vector) or ``[P, >= n]`` (one replica per worker).
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Tuple
+
+import torch
+
+OK = 0
+ERR_ARG, ERR_ALIGN, ERR_CUDA, ERR_TIMEOUT, ERR_NONFINITE, ERR_NOMEM, ERR_TOO_LARGE = -1, -2, -3, -4, -5, -6, -7
+MODE_EF = 0
+MODE_ALG1 = 1
+FORCE_TWO_PASS = 1 << 4
+FORCE_COOPERATIVE = 1 << 5
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "liba2sgd.so")
+_lib = None
+
+_vp = ctypes.c_void_p
+_i64 = ctypes.c_int64
+
+
+class A2SGDError(RuntimeError):
+    def __init__(self, status: int, what: str):
+        self.status = status
+        super().__init__(f"{what}: status {status} ({status_string(status)})")
+
+
+def lib() -> ctypes.CDLL:
+    """Loads liba2sgd.so; raises if it has not been built (no CPU fallback exists)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(
+                f"{LIB_PATH} is missing: build it with `python -m paper_2006_07405_b200.build` "
+                "(nvcc, sm_100a). This package has no CPU fallback.")
+        l = ctypes.CDLL(LIB_PATH)
+        l.a2sgd_create.restype = ctypes.c_int
+        l.a2sgd_create.argtypes = [ctypes.POINTER(_vp), ctypes.c_uint64, ctypes.c_uint32, ctypes.c_int, ctypes.c_uint32]
+        l.a2sgd_destroy.restype = ctypes.c_int
+        l.a2sgd_destroy.argtypes = [_vp]
+        l.a2sgd_encode.restype = ctypes.c_int
+        l.a2sgd_encode.argtypes = [_vp, _vp, _i64, _vp, _i64, _vp, _vp, _vp, _vp]
+        l.a2sgd_global_average.restype = ctypes.c_int
+        l.a2sgd_global_average.argtypes = [_vp, _vp, _vp, _vp]
+        l.a2sgd_decode_update.restype = ctypes.c_int
+        l.a2sgd_decode_update.argtypes = [_vp, _vp, _i64, _vp, _i64, _vp, _i64, _vp, _vp, ctypes.c_float, _vp]
+        l.a2sgd_step.restype = ctypes.c_int
+        l.a2sgd_step.argtypes = [_vp, _vp, _i64, _vp, _i64, _vp, _i64, ctypes.c_float, _vp]
+        l.a2sgd_step_host.restype = ctypes.c_int
+        l.a2sgd_step_host.argtypes = [_vp, _vp, _i64, _vp, _i64, _vp, _i64, _vp, _i64, ctypes.c_float, _vp, _vp]
+        l.a2sgd_read_stats.restype = ctypes.c_int
+        l.a2sgd_read_stats.argtypes = [_vp, _vp, _vp, _vp, ctypes.POINTER(ctypes.c_int), _vp]
+        l.a2sgd_launch_info.restype = ctypes.c_int
+        l.a2sgd_launch_info.argtypes = [_vp, _i64, ctypes.POINTER(ctypes.c_uint32)]
+        l.a2sgd_status_string.restype = ctypes.c_char_p
+        l.a2sgd_status_string.argtypes = [ctypes.c_int]
+        _lib = l
+    return _lib
+
+
+def status_string(status: int) -> str:
+    return lib().a2sgd_status_string(int(status)).decode()
+
+
+def _check(status: int, what: str) -> None:
+    if status != OK:
+        raise A2SGDError(status, what)
+
+
+def _stream(stream) -> Optional[int]:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream)
+
+
+def _rows(t: Optional[torch.Tensor], name: str) -> Tuple[Optional[int], int]:
+    """float32 CUDA [P, n] with unit inner stride -> (address, worker stride in elements)."""
+    if t is None:
+        return None, 0
+    if t.dtype != torch.float32 or not t.is_cuda or t.dim() != 2 or (t.shape[1] > 1 and t.stride(1) != 1):
+        raise ValueError(f"{name}: need a float32 CUDA tensor [P, n] with unit inner stride")
+    return t.data_ptr(), t.stride(0)
+
+
+def _weights(w: torch.Tensor) -> Tuple[int, int]:
+    if w.dtype != torch.float32 or not w.is_cuda:
+        raise ValueError("w: need a float32 CUDA tensor")
+    if w.dim() == 1:
+        return w.data_ptr(), 0
+    if w.dim() == 2:
+        return w.data_ptr(), w.stride(0)
+    raise ValueError("w: need [n] (shared) or [P, n] (replicated)")
+
+
+class Context:
+    """Owns an ``a2sgd_ctx``.  ``n`` elements per worker, ``P`` workers."""
+
+    def __init__(self, n: int, P: int, device: int = 0, flags: int = MODE_EF):
+        self.n, self.P, self.device, self.flags = int(n), int(P), int(device), int(flags)
+        self._h = _vp()
+        _check(lib().a2sgd_create(ctypes.byref(self._h), self.n, self.P, self.device, self.flags), "a2sgd_create")
+
+    @property
+    def handle(self):
+        if not self._h:
+            raise RuntimeError("context destroyed")
+        return self._h
+
+    def destroy(self) -> None:
+        if self._h:
+            lib().a2sgd_destroy(self._h)
+            self._h = _vp()
+
+    def __del__(self):
+        try:
+            self.destroy()
+        except Exception:
+            pass
+
+
+def a2sgd_create(n: int, P: int, device: int = 0, flags: int = MODE_EF) -> Context:
+    return Context(n, P, device, flags)
+
+
+def a2sgd_destroy(ctx: Context) -> None:
+    ctx.destroy()
+
+
+def a2sgd_encode(ctx: Context, grad: torch.Tensor, err: Optional[torch.Tensor], local_means: torch.Tensor,
+                 pos_counts: Optional[torch.Tensor] = None, pos_mask: Optional[torch.Tensor] = None,
+                 stream=None) -> None:
+    """local_means: float32 CUDA [P, 2]; pos_counts: int64 CUDA [P]; pos_mask: int32 CUDA [P, ceil(n/32)]."""
+    gp, gs = _rows(grad, "grad")
+    ep, es = _rows(err, "err")
+    _check(lib().a2sgd_encode(ctx.handle, gp, gs, ep, es, local_means.data_ptr(),
+                              pos_counts.data_ptr() if pos_counts is not None else None,
+                              pos_mask.data_ptr() if pos_mask is not None else None, _stream(stream)),
+           "a2sgd_encode")
+
+
+def a2sgd_global_average(ctx: Context, local_means: torch.Tensor, global_means: torch.Tensor, stream=None) -> None:
+    _check(lib().a2sgd_global_average(ctx.handle, local_means.data_ptr(), global_means.data_ptr(), _stream(stream)),
+           "a2sgd_global_average")
+
+
+def a2sgd_decode_update(ctx: Context, w: torch.Tensor, grad: torch.Tensor, err: Optional[torch.Tensor],
+                        local_means: Optional[torch.Tensor], global_means: torch.Tensor, lr: float,
+                        stream=None) -> None:
+    wp, ws = _weights(w)
+    gp, gs = _rows(grad, "grad")
+    ep, es = _rows(err, "err")
+    _check(lib().a2sgd_decode_update(ctx.handle, wp, ws, gp, gs, ep, es,
+                                     local_means.data_ptr() if local_means is not None else None,
+                                     global_means.data_ptr(), float(lr), _stream(stream)),
+           "a2sgd_decode_update")
+
+
+def a2sgd_step(ctx: Context, w: torch.Tensor, grad: torch.Tensor, err: Optional[torch.Tensor], lr: float,
+               stream=None) -> None:
+    wp, ws = _weights(w)
+    gp, gs = _rows(grad, "grad")
+    ep, es = _rows(err, "err")
+    _check(lib().a2sgd_step(ctx.handle, wp, ws, gp, gs, ep, es, float(lr), _stream(stream)), "a2sgd_step")
+
+
+def a2sgd_step_host(ctx: Context, w: torch.Tensor, grad_host: torch.Tensor, grad_staging: torch.Tensor,
+                    err: Optional[torch.Tensor], lr: float, means_host: torch.Tensor, stream=None) -> None:
+    """grad_host: float32 CPU [P, >= n] (pinned for asynchronous copies); means_host: float32 CPU [2P + 2]."""
+    if grad_host.is_cuda or grad_host.dtype != torch.float32 or grad_host.dim() != 2 or grad_host.stride(1) != 1:
+        raise ValueError("grad_host: need a float32 CPU tensor [P, n] with unit inner stride")
+    if means_host.is_cuda or means_host.dtype != torch.float32 or means_host.numel() < 2 * ctx.P + 2:
+        raise ValueError("means_host: need a float32 CPU tensor of 2P + 2 elements")
+    wp, ws = _weights(w)
+    sp, ss = _rows(grad_staging, "grad_staging")
+    ep, es = _rows(err, "err")
+    _check(lib().a2sgd_step_host(ctx.handle, wp, ws, grad_host.data_ptr(), grad_host.stride(0), sp, ss, ep, es,
+                                 float(lr), means_host.data_ptr(), _stream(stream)), "a2sgd_step_host")
+
+
+def a2sgd_read_stats(ctx: Context, stream=None):
+    """Synchronises the stream.  Returns (local_means [P,2], global_means [2], pos_counts [P], device_status)."""
+    import numpy as np
+    lm = np.zeros((ctx.P, 2), np.float32)
+    gm = np.zeros(2, np.float32)
+    pc = np.zeros(ctx.P, np.uint64)
+    st = ctypes.c_int(0)
+    _check(lib().a2sgd_read_stats(ctx.handle, lm.ctypes.data, gm.ctypes.data, pc.ctypes.data, ctypes.byref(st),
+                                  _stream(stream)), "a2sgd_read_stats")
+    return lm, gm, pc, st.value
+
+
+def a2sgd_launch_info(ctx: Context, shared_w: bool = True) -> dict:
+    out = (ctypes.c_uint32 * 5)()
+    _check(lib().a2sgd_launch_info(ctx.handle, 0 if shared_w else ctx.n, out), "a2sgd_launch_info")
+    return {"encode_ctas": out[0], "decode_ctas": out[1], "threads": out[2], "single_launch": bool(out[3]),
+            "sms": out[4]}

@@ -1,0 +1,340 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the CPU oracle on the same
+seeded inputs, element by element."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2006_07405_b200 import binding as B
+from paper_2006_07405_b200 import workloads as W
+from parity_util import assert_means, assert_state
+
+pytestmark = pytest.mark.gpu
+
+EF, ALG1 = B.MODE_EF, B.MODE_ALG1
+NAN = float("nan")
+
+
+def _state(seed, P, n, *, pad=0, off=(0, 0, 0), replicated=False, g_scale=1e-3, e_scale=3e-4):
+    """Seeded g, e, w on the GPU inside NaN-filled guard bands.  ``off`` shifts the start of
+    the g / e / w rows by that many elements (pointer misalignment); ``pad`` widens the row
+    stride beyond n.  Returns the views the library sees plus the raw buffers."""
+    rng = np.random.default_rng(seed)
+    stride = n + pad
+    raw = {}
+    views = {}
+    for k, (name, scale, rows, o) in enumerate([("g", g_scale, P, off[0]), ("e", e_scale, P, off[1]),
+                                                ("w", 0.02, P if replicated else 1, off[2])]):
+        buf = np.full(8 + o + rows * stride + 8, NAN, np.float32)
+        vals = (rng.standard_normal((rows, n)) * scale).astype(np.float32)
+        for r in range(rows):
+            buf[8 + o + r * stride: 8 + o + r * stride + n] = vals[r]
+        t = torch.from_numpy(buf).cuda()
+        raw[name] = t
+        v = t[8 + o: 8 + o + rows * stride].view(rows, stride)[:, :n]
+        views[name] = v if (name != "w" or replicated) else v[0]
+    return views, raw, stride
+
+
+def _host(views):
+    g = views["g"].cpu().numpy().copy()
+    e = views["e"].cpu().numpy().copy()
+    w = views["w"].cpu().numpy().copy()
+    return g, e, w
+
+
+def _guards_intact(raw, views, n, stride, rows_of):
+    """Everything outside the n live elements of each row is still NaN."""
+    for name, t in raw.items():
+        buf = t.cpu().numpy()
+        live = np.zeros(buf.shape, bool)
+        v = views[name]
+        start = (v.data_ptr() - t.data_ptr()) // 4
+        for r in range(rows_of[name]):
+            live[start + r * stride: start + r * stride + n] = True
+        assert np.isnan(buf[~live]).all(), f"{name}: guard band overwritten"
+        assert np.isfinite(buf[live]).all(), f"{name}: live element not finite"
+
+
+SIZES = [1, 2, 3, 4, 5, 31, 32, 33, 127, 1023, 1024, 1025, 4099, 65536 + 7, (1 << 20) - 1, (1 << 20) + 1]
+
+
+@pytest.mark.parametrize("mode", [EF, ALG1])
+@pytest.mark.parametrize("replicated", [False, True])
+@pytest.mark.parametrize("n", SIZES)
+def test_single_step_matches_oracle(mode, replicated, n):
+    P = [1, 2, 3, 4, 8, 16][(n + int(replicated)) % 6]
+    # worker stride a multiple of 4 elements (vector kernels) except when n % 3 == 0 (scalar kernels)
+    pad = ((-n) % 4) if n % 3 else 1
+    views, raw, stride = _state(1000 + n, P, n, pad=pad, replicated=replicated)
+    g, e, w = _host(views)
+    ctx = B.a2sgd_create(n, P, 0, mode)
+    # stage 1: encode (means, counts, mask) -- bit-exact integers, 1e-6 means
+    lm_buf = torch.full((P + 2, 2), NAN, device="cuda")
+    lm = lm_buf[1:P + 1]
+    cnt = torch.zeros(P, dtype=torch.int64, device="cuda")
+    words = (n + 31) // 32
+    mask = torch.zeros((P, words), dtype=torch.int32, device="cuda")
+    B.a2sgd_encode(ctx, views["g"], views["e"] if mode == EF else None, lm, cnt, mask)
+    lm_ref, cnt_ref, mask_ref = oracle.encode(g, e if mode == EF else None, mode=mode, want_mask=True)
+    assert np.array_equal(cnt.cpu().numpy().astype(np.uint64), cnt_ref)
+    assert np.array_equal(mask.cpu().numpy().view(np.uint32), mask_ref)
+    assert_means(lm.cpu().numpy(), lm_ref, "local means")
+    # payload: exactly two floats per worker were written
+    assert torch.isnan(lm_buf[0]).all() and torch.isnan(lm_buf[P + 1]).all()
+    # stage 2: global average
+    gm = torch.zeros(2, device="cuda")
+    B.a2sgd_global_average(ctx, lm, gm)
+    gm_ref = oracle.global_average(lm_ref)
+    assert_means(gm.cpu().numpy(), gm_ref, "global means")
+    # stage 3: decode / residual / SGD on copies, against the oracle's full step
+    w_staged = raw["w"].clone()
+    e_staged = raw["e"].clone()
+    w_view = w_staged[(views["w"].data_ptr() - raw["w"].data_ptr()) // 4:]
+    e_view = e_staged[(views["e"].data_ptr() - raw["e"].data_ptr()) // 4:]
+    w_arg = w_view[:P * stride].view(P, stride)[:, :n] if replicated else w_view[:n]
+    e_arg = e_view[:P * stride].view(P, stride)[:, :n]
+    B.a2sgd_decode_update(ctx, w_arg, views["g"], e_arg, lm, gm, 0.1)
+    w_ref, e_ref = w.copy(), e.copy()
+    lm_o, gm_o, cnt_o = oracle.step(w_ref, g, e_ref, 0.1, mode=mode)
+    assert_state(w_arg.cpu().numpy(), w_ref, e_arg.cpu().numpy(), e_ref, gm_o, f"staged n={n} P={P}")
+    # fused step on the originals: same bits as the staged calls
+    B.a2sgd_step(ctx, views["w"], views["g"], views["e"], 0.1)
+    lm_s, gm_s, cnt_s, status = B.a2sgd_read_stats(ctx)
+    assert status == B.OK
+    assert np.array_equal(cnt_s, cnt_ref)
+    assert np.array_equal(lm_s, lm.cpu().numpy()) and np.array_equal(gm_s, gm.cpu().numpy())
+    assert torch.equal(views["w"], w_arg) and torch.equal(views["e"], e_arg)
+    rows = {"g": P, "e": P, "w": P if replicated else 1}
+    _guards_intact(raw, views, n, stride, rows)
+    # the gradient is never written
+    assert np.array_equal(views["g"].cpu().numpy(), g)
+    ctx.destroy()
+
+
+@pytest.mark.parametrize("mode", [EF, ALG1])
+@pytest.mark.parametrize("off", [(1, 0, 0), (0, 1, 0), (0, 0, 1), (1, 2, 3), (3, 3, 3), (2, 0, 2)])
+def test_misaligned_pointers(mode, off):
+    n, P = 10007, 3
+    for replicated in (False, True):
+        views, raw, stride = _state(77, P, n, pad=3, off=off, replicated=replicated)
+        g, e, w = _host(views)
+        ctx = B.a2sgd_create(n, P, 0, mode)
+        B.a2sgd_step(ctx, views["w"], views["g"], views["e"], 0.05)
+        lm, gm, cnt, status = B.a2sgd_read_stats(ctx)
+        lm_ref, gm_ref, cnt_ref = oracle.step(w, g, e, 0.05, mode=mode)
+        assert status == B.OK and np.array_equal(cnt, cnt_ref)
+        assert_means(lm, lm_ref)
+        assert_means(gm, gm_ref)
+        assert_state(views["w"].cpu().numpy(), w, views["e"].cpu().numpy(), e, gm_ref, f"off={off}")
+        _guards_intact(raw, views, n, stride, {"g": P, "e": P, "w": P if replicated else 1})
+        ctx.destroy()
+
+
+def test_alg1_without_error_buffer_and_single_worker_is_dense_sgd():
+    n = 50001
+    views, raw, stride = _state(5, 1, n)
+    g, e, w = _host(views)
+    ctx = B.a2sgd_create(n, 1, 0, ALG1)
+    B.a2sgd_step(ctx, views["w"], views["g"], None, 0.1)
+    torch.cuda.synchronize()
+    # P = 1: Algorithm 1 returns g itself, the update is one fp32 fma per element
+    ref = w.astype(np.float64) - np.float64(np.float32(0.1)) * g[0].astype(np.float64)
+    got = views["w"].cpu().numpy()
+    assert np.max(np.abs(got - ref)) <= np.spacing(np.abs(w).max())
+    assert np.array_equal(views["e"].cpu().numpy(), e)   # untouched when no err pointer is passed
+    ctx.destroy()
+
+
+@pytest.mark.parametrize("case", ["all_pos", "all_neg", "zeros", "neg_zero", "subnormal", "two_valued"])
+def test_degenerate_inputs(case):
+    n, P = 3001, 2
+    views, raw, stride = _state(9, P, n)
+    g = views["g"]
+    views["e"].zero_()
+    if case == "all_pos":
+        g.abs_()
+    elif case == "all_neg":
+        g.abs_().neg_().sub_(1e-9)
+    elif case == "zeros":
+        g.zero_()
+    elif case == "neg_zero":
+        g.zero_().neg_()
+    elif case == "subnormal":
+        g.copy_(torch.where(g >= 0, torch.full_like(g, 1e-45), torch.full_like(g, -1e-45)))
+    elif case == "two_valued":
+        g.copy_(torch.where(g >= 0, torch.full_like(g, 0.75), torch.full_like(g, -0.125)))
+    gh, eh, wh = _host(views)
+    ctx = B.a2sgd_create(n, P, 0, EF)
+    lm = torch.zeros((P, 2), device="cuda")
+    cnt = torch.zeros(P, dtype=torch.int64, device="cuda")
+    mask = torch.zeros((P, (n + 31) // 32), dtype=torch.int32, device="cuda")
+    B.a2sgd_encode(ctx, views["g"], views["e"], lm, cnt, mask)
+    lm_ref, cnt_ref, mask_ref = oracle.encode(gh, eh, mode=EF, want_mask=True)
+    assert np.array_equal(cnt.cpu().numpy().astype(np.uint64), cnt_ref)
+    assert np.array_equal(mask.cpu().numpy().view(np.uint32), mask_ref)
+    if case in ("all_pos", "all_neg"):
+        assert_means(lm.cpu().numpy(), lm_ref)
+    else:
+        assert np.array_equal(lm.cpu().numpy(), lm_ref)  # sums of these values are exact in fp32
+    B.a2sgd_step(ctx, views["w"], views["g"], views["e"], 0.1)
+    oracle.step(wh, gh, eh, 0.1, mode=EF)
+    _, gm, _, status = B.a2sgd_read_stats(ctx)
+    assert status == B.OK
+    assert_state(views["w"].cpu().numpy(), wh, views["e"].cpu().numpy(), eh, gm, case)
+    if case == "two_valued":
+        assert not views["e"].any()
+    ctx.destroy()
+
+
+def test_run_to_run_bitwise_reproducible():
+    wl = W.scaled(W.get_workload("c3_resnet50"), 8)
+    n, P = wl.n, wl.P
+    g = torch.empty((P, n), device="cuda")
+    W.fill_gradients(wl, 0, g)
+    e0 = torch.randn((P, n), device="cuda", generator=torch.Generator("cuda").manual_seed(3)) * 1e-4
+    w0 = torch.empty(n, device="cuda")
+    W.init_weights(wl, w0)
+    outs = []
+    for _ in range(3):
+        ctx = B.a2sgd_create(n, P, 0, EF)
+        e, w = e0.clone(), w0.clone()
+        B.a2sgd_step(ctx, w, g, e, wl.lr)
+        lm, gm, cnt, _ = B.a2sgd_read_stats(ctx)
+        outs.append((lm.tobytes(), gm.tobytes(), cnt.tobytes(), e.cpu().numpy().tobytes(), w.cpu().numpy().tobytes()))
+        ctx.destroy()
+    assert outs[0] == outs[1] == outs[2]
+
+
+@pytest.mark.parametrize("name,div", [("c1_flat_1m", 1), ("c2_lstm_ptb", 16), ("c3_resnet50", 4),
+                                      ("c4_vgg16", 32), ("c5_gpt2_xl", 256)])
+@pytest.mark.parametrize("mode", [EF, ALG1])
+def test_free_running_multi_step(name, div, mode):
+    """The benchmark configurations (tensor structure kept, lengths divided so that the oracle
+    finishes in seconds), run for their stated number of steps, GPU and oracle each on its own
+    evolving state."""
+    wl = W.get_workload(name)
+    wl = W.scaled(wl, div) if div > 1 else wl
+    n, P = wl.n, wl.P
+    g = torch.empty((P, n), device="cuda")
+    e = torch.zeros((P, n), device="cuda")
+    w = torch.empty(n, device="cuda")
+    W.init_weights(wl, w)
+    e_ref = np.zeros((P, n), np.float32)
+    w_ref = w.cpu().numpy().copy()
+    ctx = B.a2sgd_create(n, P, 0, mode)
+    flips = 0
+    for step in range(wl.steps):
+        W.fill_gradients(wl, step, g)
+        gh = g.cpu().numpy()
+        B.a2sgd_step(ctx, w, g, e, wl.lr)
+        lm, gm, cnt, status = B.a2sgd_read_stats(ctx)
+        lm_ref, gm_ref, cnt_ref = oracle.step(w_ref, gh, e_ref, wl.lr, mode=mode)
+        assert status == B.OK
+        # from step 2 on the two error buffers differ by rounding, so an element whose
+        # compensated value sits at rounding level may change group: count, do not fail
+        flips += int(np.abs(cnt.astype(np.int64) - cnt_ref.astype(np.int64)).sum())
+        if step == 0:
+            assert np.array_equal(cnt, cnt_ref)
+        assert_means(lm, lm_ref, f"{name} step {step} local means")
+        assert_means(gm, gm_ref, f"{name} step {step} global means")
+        allowed = 0 if step == 0 else max(2, n * P // 1_000_000)
+        assert_state(w.cpu().numpy(), w_ref, e.cpu().numpy(), e_ref, gm_ref, f"{name} step {step}",
+                     max_outliers=allowed)
+    assert flips <= max(2, n * P // 1_000_000), f"{flips} group changes"
+    ctx.destroy()
+
+
+def test_nonfinite_input_is_latched_in_status_word():
+    n, P = 5000, 2
+    views, raw, stride = _state(21, P, n)
+    views["g"][1, 1234] = float("inf")
+    ctx = B.a2sgd_create(n, P, 0, EF)
+    lm = torch.zeros((P, 2), device="cuda")
+    B.a2sgd_encode(ctx, views["g"], views["e"], lm)
+    *_, status = B.a2sgd_read_stats(ctx)
+    assert status == B.ERR_NONFINITE
+    *_, status = B.a2sgd_read_stats(ctx)
+    assert status == B.OK          # the latch is cleared by the read
+    ctx.destroy()
+
+
+def test_bad_arguments_return_status_and_launch_nothing():
+    n, P = 1000, 2
+    views, raw, stride = _state(22, P, n)
+    before = {k: v.clone() for k, v in raw.items()}
+    with pytest.raises(B.A2SGDError) as ei:
+        B.a2sgd_create(0, 1)
+    assert ei.value.status == B.ERR_ARG
+    with pytest.raises(B.A2SGDError):
+        B.a2sgd_create(10, 0)
+    with pytest.raises(B.A2SGDError):
+        B.a2sgd_create(10, 1025)
+    with pytest.raises(B.A2SGDError):
+        B.a2sgd_create(10, 1, 0, 1 << 20)
+    with pytest.raises(B.A2SGDError):
+        B.a2sgd_create(10, 1, 99)
+    ctx = B.a2sgd_create(n, P, 0, EF)
+    with pytest.raises(B.A2SGDError) as ei:
+        B.a2sgd_step(ctx, views["w"], views["g"], None, 0.1)       # EF needs err
+    assert ei.value.status == B.ERR_ARG
+    with pytest.raises(B.A2SGDError) as ei:                          # worker stride < n
+        B.a2sgd_step(ctx, views["w"], views["g"][:, : n // 2].contiguous().view(P, n // 2), views["e"], 0.1)
+    assert ei.value.status == B.ERR_ARG
+    h = ctx.handle
+    st = B.lib().a2sgd_step(h, views["w"].data_ptr() + 2, 0, views["g"].data_ptr(), stride,
+                            views["e"].data_ptr(), stride, 0.1, None)
+    assert st == B.ERR_ALIGN
+    torch.cuda.synchronize()
+    for k in raw:
+        assert torch.equal(torch.nan_to_num(raw[k]), torch.nan_to_num(before[k]))
+    assert "argument" in B.status_string(B.ERR_ARG)
+    ctx.destroy()
+
+
+def test_checkpoint_resume_is_bitwise():
+    """All state is caller-owned: 5 steps == 3 steps, copy out / in, new context, 2 steps."""
+    wl = W.scaled(W.get_workload("c2_lstm_ptb"), 64)
+    n, P = wl.n, wl.P
+    g = torch.empty((P, n), device="cuda")
+
+    def run(split):
+        e = torch.zeros((P, n), device="cuda")
+        w = torch.empty(n, device="cuda")
+        W.init_weights(wl, w)
+        ctx = B.a2sgd_create(n, P, 0, EF)
+        for step in range(5):
+            if step == split:
+                e = e.cpu().cuda()
+                w = w.cpu().cuda()
+                ctx.destroy()
+                ctx = B.a2sgd_create(n, P, 0, EF)
+            W.fill_gradients(wl, step, g)
+            B.a2sgd_step(ctx, w, g, e, wl.lr)
+        torch.cuda.synchronize()
+        return e.cpu(), w.cpu()
+
+    ea, wa = run(None)
+    eb, wb = run(3)
+    assert torch.equal(ea, eb) and torch.equal(wa, wb)
+
+
+def test_host_gradient_entry_point():
+    wl = W.scaled(W.get_workload("c2_lstm_ptb"), 32)
+    n, P = wl.n, wl.P
+    g_host = torch.empty((P, n)).pin_memory()
+    W.fill_gradients(wl, 0, g_host)
+    staging = torch.empty((P, n), device="cuda")
+    e = torch.zeros((P, n), device="cuda")
+    w = torch.empty(n, device="cuda")
+    W.init_weights(wl, w)
+    w_ref = w.cpu().numpy().copy()
+    e_ref = np.zeros((P, n), np.float32)
+    means = torch.zeros(2 * P + 2).pin_memory()
+    ctx = B.a2sgd_create(n, P, 0, EF)
+    B.a2sgd_step_host(ctx, w, g_host, staging, e, wl.lr, means)
+    lm_ref, gm_ref, _ = oracle.step(w_ref, g_host.numpy(), e_ref, wl.lr, mode=EF)
+    assert_means(means[:2 * P].numpy().reshape(P, 2), lm_ref)
+    assert_means(means[2 * P:].numpy(), gm_ref)
+    assert_state(w.cpu().numpy(), w_ref, e.cpu().numpy(), e_ref, gm_ref, "host entry")
+    ctx.destroy()
