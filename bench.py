@@ -194,8 +194,9 @@ def time_workload(wl, steps, warmup, dev, *, with_roofline=True, with_e2e=True, 
 
     n, P = wl.n, wl.P
     torch.cuda.set_device(dev)
-    g = torch.empty((P, n), device=dev)
-    e = torch.zeros((P, n), device=dev)
+    # rows start 128-byte aligned (row stride = n rounded up to 32 elements)
+    g = B.padded_rows(P, n, dev)
+    e = B.padded_rows(P, n, dev, fill=0.0)
     w = torch.empty(n, device=dev)
     W.fill_gradients(wl, 0, g)
     W.init_weights(wl, w)
@@ -212,11 +213,34 @@ def time_workload(wl, steps, warmup, dev, *, with_roofline=True, with_e2e=True, 
     for _ in range(max(warmup, 3)):
         B.a2sgd_step(ctx, w, g, e, wl.lr)
     barrier()
+    # A step of a few microseconds is bound by host launch overhead: replay it from a CUDA graph
+    # (chunks of `chunk` steps, K = reps * chunk exactly).
+    graph, chunk = None, 1
+    if n * P < (1 << 23):
+        chunk = max(d for d in range(1, 51) if steps % d == 0)
+        try:
+            side = torch.cuda.Stream(dev)
+            side.wait_stream(torch.cuda.current_stream(dev))
+            with torch.cuda.stream(side):
+                graph = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(graph, stream=side):
+                    for _ in range(chunk):
+                        B.a2sgd_step(ctx, w, g, e, wl.lr, stream=side)
+            torch.cuda.current_stream(dev).wait_stream(side)
+            graph.replay()
+        except Exception as ex:  # capture refused: time eager launches instead
+            graph, chunk = None, 1
+            sys.stderr.write(f"CUDA graph capture failed ({ex}); timing eager launches\n")
+        barrier()
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     wall0 = time.time()
     ev0.record()
-    for _ in range(steps):
-        B.a2sgd_step(ctx, w, g, e, wl.lr)
+    if graph is not None:
+        for _ in range(steps // chunk):
+            graph.replay()
+    else:
+        for _ in range(steps):
+            B.a2sgd_step(ctx, w, g, e, wl.lr)
     ev1.record()
     barrier()
     wall1 = time.time()
@@ -226,7 +250,9 @@ def time_workload(wl, steps, warmup, dev, *, with_roofline=True, with_e2e=True, 
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
         ms = float(t.item())
     res = {"ms_total": ms, "ms_per_step": ms / steps, "launches": launches_per_step * steps,
-           "launch_info": info, "wall": (wall0, wall1)}
+           "launch_info": info, "wall": (wall0, wall1),
+           "launch_mode": f"CUDA graph of {chunk} steps" if graph is not None else "eager"}
+    del graph
     *_, status = B.a2sgd_read_stats(ctx)
     res["device_status"] = status
 
@@ -289,8 +315,8 @@ def load_loop_for_clocks(wl, dev, seconds):
     from paper_2006_07405_b200 import binding as B
     from paper_2006_07405_b200 import workloads as W
     n, P = wl.n, wl.P
-    g = torch.empty((P, n), device=dev)
-    e = torch.zeros((P, n), device=dev)
+    g = B.padded_rows(P, n, dev)
+    e = B.padded_rows(P, n, dev, fill=0.0)
     w = torch.zeros(n, device=dev)
     W.fill_gradients(wl, 0, g)
     ctx = B.a2sgd_create(n, P, dev.index, B.MODE_EF)
@@ -305,7 +331,8 @@ def load_loop_for_clocks(wl, dev, seconds):
 def summarise(wl, res, n_gpus, peak_gbs):
     b = algorithmic_bytes_per_model_element(wl.P)
     t = res["ms_per_step"] * 1e-3
-    out = {"n": wl.n, "P": wl.P, "ms_per_step": res["ms_per_step"],
+    out = {"n": wl.n, "P": wl.P, "ms_per_step": res["ms_per_step"], "launch_mode": res["launch_mode"],
+           "single_launch": res["launch_info"]["single_launch"],
            "model_params_per_s": n_gpus * wl.n / t, "worker_params_per_s": n_gpus * wl.n * wl.P / t,
            "step_GBps": b["step"] * wl.n / t / 1e9,
            "step_frac_of_8TBps": b["step"] * wl.n / t / 1e9 / NOMINAL_HBM_GBS,
@@ -327,6 +354,11 @@ def main():
     ap.add_argument("--impl", default="native", choices=["native", "reference"])
     ap.add_argument("--no-extra", action="store_true", help="skip the extra c4/c5 measurements at N=1")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--scale-div", type=int, default=1,
+                    help="divide every tensor length of the workload (small cases for profiler captures)")
+    ap.add_argument("--minimal", action="store_true",
+                    help="timed step loop only (for profiler captures): no e2e, no per-kernel loop, "
+                         "no extra workloads, no clock load loop, no CPU baseline")
     args = ap.parse_args()
 
     if args.impl == "reference":
@@ -354,9 +386,20 @@ def main():
     dev = torch.device("cuda", local_rank)
     torch.cuda.set_device(dev)
     wl = W.get_workload(args.workload)
+    if args.scale_div > 1:
+        wl = W.scaled(wl, args.scale_div)
     peak_gbs, peak_src = measured_peak_gbs()
     steps, warmup = max(1, args.steps), max(3, args.warmup)
 
+    if args.minimal:
+        res = time_workload(wl, steps, warmup, dev, with_roofline=False, with_e2e=False, dist=dist)
+        if rank == 0:
+            print(json.dumps({"metric": METRIC, "value": n_gpus * wl.n / (res["ms_per_step"] * 1e-3), "unit": UNIT,
+                              "ms_per_step": res["ms_per_step"], "steps": steps, "warmup": warmup,
+                              "config": W.describe(wl), "note": "minimal run for profiler captures"}), flush=True)
+        if dist is not None:
+            dist.destroy_process_group()
+        return
     sampler = ClockSampler(local_rank) if rank == 0 else None
     res = time_workload(wl, steps, warmup, dev, dist=dist)
     if rank == 0 and res["ms_total"] < 1500.0:
@@ -367,7 +410,7 @@ def main():
             "timed region plus 1.5 s of the same step loop (timed region shorter than the sampling period allows)"
 
     extra = {}
-    if rank == 0 and world == 1 and not args.no_extra and args.workload == "c2_lstm_ptb":
+    if rank == 0 and world == 1 and not args.no_extra and args.workload == "c2_lstm_ptb" and args.scale_div == 1:
         free_b, _ = torch.cuda.mem_get_info(dev)
         for name in ("c1_flat_1m", "c3_resnet50", "c4_vgg16", "c5_gpt2_xl"):
             w2 = W.get_workload(name)
@@ -403,7 +446,8 @@ def main():
                        step_GBps=b["step"] * wl.n / t / 1e9,
                        step_frac_of_8TBps=b["step"] * wl.n / t / 1e9 / NOMINAL_HBM_GBS,
                        step_frac_of_measured_peak=b["step"] * wl.n / t / 1e9 / peak_gbs,
-                       bytes_per_model_element=b, launch=res["launch_info"],
+                       bytes_per_model_element=b, launch=res["launch_info"], launch_mode=res["launch_mode"],
+                       row_stride="n rounded up to 32 elements (rows start 128-byte aligned)",
                        encode_ms=res["encode_ms"], decode_ms=res["decode_ms"],
                        device_status=res["device_status"]),
         "gpu_launches": res["launches"],

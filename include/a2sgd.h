@@ -72,7 +72,10 @@ enum a2sgd_flags {
     A2SGD_MODE_EF = 0,                /* default */
     A2SGD_MODE_ALG1 = 1,
     A2SGD_FORCE_TWO_PASS = 1 << 4,    /* a2sgd_step never takes the single-launch path */
-    A2SGD_FORCE_COOPERATIVE = 1 << 5  /* a2sgd_step always takes it; A2SGD_ERR_TOO_LARGE if it cannot */
+    A2SGD_FORCE_COOPERATIVE = 1 << 5, /* a2sgd_step always takes it; A2SGD_ERR_TOO_LARGE if it cannot */
+    A2SGD_TEST_BARRIER_NEVER_OPENS = 1 << 9 /* test hook: the single-launch path waits for one arrival more
+                                               than its grid has, with a ~0.2 ms limit, so every CTA gives up,
+                                               writes nothing and A2SGD_ERR_TIMEOUT is latched */
 };
 
 /* Creates a context for vectors of n elements and P workers on `device`

@@ -23,6 +23,8 @@ MODE_EF = 0
 MODE_ALG1 = 1
 FORCE_TWO_PASS = 1 << 4
 FORCE_COOPERATIVE = 1 << 5
+TEST_BARRIER_NEVER_OPENS = 1 << 9
+ROW_ALIGN_ELEMS = 32   # 128 bytes: rows that start on a cache-line boundary take the widest vector kernels
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "liba2sgd.so")
@@ -103,6 +105,16 @@ def _weights(w: torch.Tensor) -> Tuple[int, int]:
     if w.dim() == 2:
         return w.data_ptr(), w.stride(0)
     raise ValueError("w: need [n] (shared) or [P, n] (replicated)")
+
+
+def padded_rows(P: int, n: int, device, fill: Optional[float] = None) -> torch.Tensor:
+    """A float32 [P, n] view whose rows start 128-byte aligned (row stride = n rounded up to 32
+    elements).  Device memory only; the layout the fast kernels are measured with."""
+    stride = (n + ROW_ALIGN_ELEMS - 1) // ROW_ALIGN_ELEMS * ROW_ALIGN_ELEMS
+    buf = torch.empty((P, stride), dtype=torch.float32, device=device)
+    if fill is not None:
+        buf.fill_(fill)
+    return buf[:, :n]
 
 
 class Context:

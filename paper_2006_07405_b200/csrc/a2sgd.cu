@@ -7,10 +7,15 @@
 #include <algorithm>
 #include <cstdint>
 #include <new>
+#include <unordered_map>
 
 #include "a2sgd_kernels.cuh"
 
 using namespace a2sgd;
+
+#ifndef A2SGD_MAX_VW
+#define A2SGD_MAX_VW 8 /* widest vector access the dispatcher may pick: 8 = 256-bit, 4 = 128-bit */
+#endif
 
 struct a2sgd_ctx {
     uint64_t n = 0;
@@ -19,6 +24,7 @@ struct a2sgd_ctx {
     uint32_t flags = 0;
     bool alg1 = false;
     int sm_count = 0;
+    bool coop_supported = false;
     // scratch (device)
     Partial *partials = nullptr;
     uint32_t g_alloc = 0; // CTAs per worker the partials array can hold
@@ -26,11 +32,11 @@ struct a2sgd_ctx {
     float *global_means = nullptr;
     unsigned long long *pos_counts = nullptr;
     unsigned int *tickets = nullptr;
+    unsigned int *barrier = nullptr; // 2 words: arrival counter, release epoch
     int *status = nullptr;
-    // resident CTAs per SM of each kernel family (occupancy API, queried once)
-    int occ_encode = 0;
-    int occ_decode_shared = 0;
-    int occ_decode_repl = 0;
+    unsigned int coop_epoch = 0;
+    // resident CTAs per SM of every kernel instance used so far (occupancy API, cached)
+    std::unordered_map<const void *, int> occ;
 };
 
 namespace {
@@ -66,10 +72,27 @@ inline bool stride_ok(int64_t stride, uint64_t n, uint32_t P)
     return P == 1 || (stride >= 0 && (uint64_t)stride >= n);
 }
 
-// 16-byte aligned base and (for P > 1) worker stride a multiple of 4 elements
-inline bool vec_ok(const void *p, int64_t stride, uint32_t P)
+// Widest vector access (elements) this pointer / worker stride allows: 8, 4 or 0 (scalar).
+inline int vec_width(const void *p, int64_t stride, uint32_t P)
 {
-    return p == nullptr || (aligned(p, 16) && (P == 1 || stride % 4 == 0));
+    if (p == nullptr) return 8;
+    if (A2SGD_MAX_VW >= 8 && aligned(p, 32) && (P == 1 || stride % 8 == 0)) return 8;
+    if (aligned(p, 16) && (P == 1 || stride % 4 == 0)) return 4;
+    return 0;
+}
+
+int occupancy(a2sgd_ctx *c, const void *kernel)
+{
+    auto it = c->occ.find(kernel);
+    if (it != c->occ.end()) return it->second;
+    int occ = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kernel, kBlock, 0) != cudaSuccess) {
+        (void)cudaGetLastError();
+        occ = 1;
+    }
+    occ = std::max(occ, 1);
+    c->occ[kernel] = occ;
+    return occ;
 }
 
 // CTAs per worker for a (G, P) grid that fills the device exactly once.
@@ -89,28 +112,83 @@ inline uint32_t flat_grid(const a2sgd_ctx *c, int occ, uint64_t items)
     return (uint32_t)std::min(slots, need);
 }
 
-template <typename K>
-int occupancy(K kernel)
+// ---------------------------------------------------------------- kernel selection
+const void *select_encode(bool ef, bool mask, int vw)
 {
-    int occ = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kernel, kBlock, 0) != cudaSuccess) {
-        (void)cudaGetLastError();
-        return 1;
+#define A2_PICK(EF, MASK)                                                               \
+    (vw == 8 ? (const void *)k_encode_vec<EF, MASK, 8>                                  \
+             : vw == 4 ? (const void *)k_encode_vec<EF, MASK, 4> : (const void *)k_encode_scalar<EF, MASK>)
+    if (ef) return mask ? A2_PICK(true, true) : A2_PICK(true, false);
+    return mask ? A2_PICK(false, true) : A2_PICK(false, false);
+#undef A2_PICK
+}
+
+template <bool EF, bool STORE, int VW>
+const void *select_decode_shared_p(uint32_t P)
+{
+    switch (P) {
+    case 1: return (const void *)k_decode_shared_vec<EF, STORE, 1, VW>;
+    case 2: return (const void *)k_decode_shared_vec<EF, STORE, 2, VW>;
+    case 4: return (const void *)k_decode_shared_vec<EF, STORE, 4, VW>;
+    case 8: return (const void *)k_decode_shared_vec<EF, STORE, 8, VW>;
+    default: return (const void *)k_decode_shared_vec<EF, STORE, 0, VW>;
     }
-    return std::max(occ, 1);
+}
+
+const void *select_decode_shared(bool ef, bool store, uint32_t P, int vw)
+{
+    if (vw == 8) {
+        if (ef) return select_decode_shared_p<true, true, 8>(P);
+        return store ? select_decode_shared_p<false, true, 8>(P) : select_decode_shared_p<false, false, 8>(P);
+    }
+    if (ef) return select_decode_shared_p<true, true, 4>(P);
+    return store ? select_decode_shared_p<false, true, 4>(P) : select_decode_shared_p<false, false, 4>(P);
+}
+
+const void *select_decode_repl(bool ef, bool store, int vw)
+{
+    if (vw == 8) {
+        if (ef) return (const void *)k_decode_repl_vec<true, true, 8>;
+        return store ? (const void *)k_decode_repl_vec<false, true, 8> : (const void *)k_decode_repl_vec<false, false, 8>;
+    }
+    if (ef) return (const void *)k_decode_repl_vec<true, true, 4>;
+    return store ? (const void *)k_decode_repl_vec<false, true, 4> : (const void *)k_decode_repl_vec<false, false, 4>;
+}
+
+const void *select_decode_scalar(bool ef, bool store)
+{
+    if (ef) return (const void *)k_decode_scalar<true, true>;
+    return store ? (const void *)k_decode_scalar<false, true> : (const void *)k_decode_scalar<false, false>;
+}
+
+template <bool EF, bool STORE, bool SHARED>
+const void *select_coop_p(uint32_t P)
+{
+    switch (P) {
+    case 1: return (const void *)k_step_coop<EF, STORE, 1, SHARED>;
+    case 2: return (const void *)k_step_coop<EF, STORE, 2, SHARED>;
+    case 4: return (const void *)k_step_coop<EF, STORE, 4, SHARED>;
+    case 8: return (const void *)k_step_coop<EF, STORE, 8, SHARED>;
+    default: return nullptr;
+    }
+}
+
+const void *select_coop(bool ef, bool store, bool shared, uint32_t P)
+{
+    if (ef) return shared ? select_coop_p<true, true, true>(P) : select_coop_p<true, true, false>(P);
+    if (store) return shared ? select_coop_p<false, true, true>(P) : select_coop_p<false, true, false>(P);
+    return shared ? select_coop_p<false, false, true>(P) : select_coop_p<false, false, false>(P);
 }
 
 // ---------------------------------------------------------------- launches
-int launch_encode(a2sgd_ctx *c, const float *grad, int64_t gs, const float *err, int64_t es,
-                  float *local_means, unsigned long long *pos_counts, uint32_t *pos_mask,
-                  float *global_means, cudaStream_t s)
+EncodeArgs make_encode_args(a2sgd_ctx *c, const float *grad, int64_t gs, const float *err, int64_t es,
+                            float *local_means, unsigned long long *pos_counts, uint32_t *pos_mask,
+                            float *global_means)
 {
-    const bool ef = !c->alg1;
-    const bool vec = vec_ok(grad, gs, c->P) && (!ef || vec_ok(err, es, c->P));
     EncodeArgs a{};
     a.grad = grad;
     a.grad_stride = gs;
-    a.err = ef ? err : nullptr;
+    a.err = c->alg1 ? nullptr : err;
     a.err_stride = es;
     a.n = c->n;
     a.P = c->P;
@@ -123,43 +201,12 @@ int launch_encode(a2sgd_ctx *c, const float *grad, int64_t gs, const float *err,
     a.global_means = global_means;
     a.ctx_local_means = c->local_means;
     a.ctx_pos_counts = c->pos_counts;
-    const uint64_t items = vec ? (c->n + 3) / 4 : c->n;
-    const dim3 grid(per_worker_grid(c, c->occ_encode, items), c->P);
-    const bool mask = pos_mask != nullptr;
-#define A2_ENC(KERNEL)                                                      \
-    do {                                                                    \
-        if (ef && mask) KERNEL<true, true><<<grid, kBlock, 0, s>>>(a);      \
-        else if (ef) KERNEL<true, false><<<grid, kBlock, 0, s>>>(a);        \
-        else if (mask) KERNEL<false, true><<<grid, kBlock, 0, s>>>(a);      \
-        else KERNEL<false, false><<<grid, kBlock, 0, s>>>(a);               \
-    } while (0)
-    if (vec) A2_ENC(k_encode_vec);
-    else A2_ENC(k_encode_scalar);
-#undef A2_ENC
-    A2_CUDA(cudaGetLastError());
-    return A2SGD_OK;
+    return a;
 }
 
-template <bool EF, bool STORE>
-void launch_decode_shared(const DecodeArgs &a, uint32_t grid, cudaStream_t s)
+DecodeArgs make_decode_args(a2sgd_ctx *c, float *w, int64_t ws, const float *grad, int64_t gs, float *err,
+                            int64_t es, const float *local_means, const float *global_means, float lr)
 {
-    switch (a.P) {
-    case 1: k_decode_shared_vec<EF, STORE, 1><<<grid, kBlock, 0, s>>>(a); break;
-    case 2: k_decode_shared_vec<EF, STORE, 2><<<grid, kBlock, 0, s>>>(a); break;
-    case 4: k_decode_shared_vec<EF, STORE, 4><<<grid, kBlock, 0, s>>>(a); break;
-    case 8: k_decode_shared_vec<EF, STORE, 8><<<grid, kBlock, 0, s>>>(a); break;
-    default: k_decode_shared_vec<EF, STORE, 0><<<grid, kBlock, 0, s>>>(a); break;
-    }
-}
-
-int launch_decode(a2sgd_ctx *c, float *w, int64_t ws, const float *grad, int64_t gs, float *err,
-                  int64_t es, const float *local_means, const float *global_means, float lr,
-                  cudaStream_t s)
-{
-    const bool ef = !c->alg1;
-    const bool store = ef || err != nullptr;
-    const bool shared = ws == 0;
-    const bool vec = vec_ok(grad, gs, c->P) && vec_ok(err, es, c->P) && vec_ok(w, shared ? 4 : ws, c->P);
     DecodeArgs a{};
     a.w = w;
     a.w_stride = ws;
@@ -172,24 +219,97 @@ int launch_decode(a2sgd_ctx *c, float *w, int64_t ws, const float *grad, int64_t
     a.local_means = local_means;
     a.global_means = global_means;
     a.lr = lr;
-    if (vec && shared) {
-        const uint32_t grid = flat_grid(c, c->occ_decode_shared, (c->n + 3) / 4);
-        if (ef) launch_decode_shared<true, true>(a, grid, s);
-        else if (store) launch_decode_shared<false, true>(a, grid, s);
-        else launch_decode_shared<false, false>(a, grid, s);
-    } else if (vec) {
-        const dim3 grid(per_worker_grid(c, c->occ_decode_repl, (c->n + 3) / 4), c->P);
-        if (ef) k_decode_repl_vec<true, true><<<grid, kBlock, 0, s>>>(a);
-        else if (store) k_decode_repl_vec<false, true><<<grid, kBlock, 0, s>>>(a);
-        else k_decode_repl_vec<false, false><<<grid, kBlock, 0, s>>>(a);
+    return a;
+}
+
+int encode_vec_width(const a2sgd_ctx *c, const float *grad, int64_t gs, const float *err, int64_t es)
+{
+    int vw = vec_width(grad, gs, c->P);
+    if (!c->alg1) vw = std::min(vw, vec_width(err, es, c->P));
+    return vw;
+}
+
+int decode_vec_width(const a2sgd_ctx *c, const float *w, int64_t ws, const float *grad, int64_t gs,
+                     const float *err, int64_t es)
+{
+    int vw = std::min(vec_width(grad, gs, c->P), vec_width(err, es, c->P));
+    return std::min(vw, vec_width(w, ws == 0 ? 8 : ws, c->P));
+}
+
+int launch_encode(a2sgd_ctx *c, const float *grad, int64_t gs, const float *err, int64_t es,
+                  float *local_means, unsigned long long *pos_counts, uint32_t *pos_mask,
+                  float *global_means, cudaStream_t s)
+{
+    const int vw = encode_vec_width(c, grad, gs, err, es);
+    EncodeArgs a = make_encode_args(c, grad, gs, err, es, local_means, pos_counts, pos_mask, global_means);
+    const void *fn = select_encode(!c->alg1, pos_mask != nullptr, vw);
+    const uint64_t items = vw ? (c->n + vw - 1) / vw : c->n;
+    const dim3 grid(per_worker_grid(c, occupancy(c, fn), items), c->P);
+    void *params[] = {&a};
+    A2_CUDA(cudaLaunchKernel(fn, grid, dim3(kBlock), params, 0, s));
+    return A2SGD_OK;
+}
+
+int launch_decode(a2sgd_ctx *c, float *w, int64_t ws, const float *grad, int64_t gs, float *err,
+                  int64_t es, const float *local_means, const float *global_means, float lr,
+                  cudaStream_t s)
+{
+    const bool ef = !c->alg1;
+    const bool store = ef || err != nullptr;
+    const bool shared = ws == 0;
+    const int vw = decode_vec_width(c, w, ws, grad, gs, err, es);
+    DecodeArgs a = make_decode_args(c, w, ws, grad, gs, err, es, local_means, global_means, lr);
+    void *params[] = {&a};
+    const void *fn;
+    dim3 grid;
+    if (vw && shared) {
+        fn = select_decode_shared(ef, store, c->P, vw);
+        grid = dim3(flat_grid(c, occupancy(c, fn), (c->n + vw - 1) / vw));
+    } else if (vw) {
+        fn = select_decode_repl(ef, store, vw);
+        grid = dim3(per_worker_grid(c, occupancy(c, fn), (c->n + vw - 1) / vw), c->P);
     } else {
-        const dim3 grid = shared ? dim3(flat_grid(c, 8, c->n), 1)
-                                 : dim3(per_worker_grid(c, 8, c->n), c->P);
-        if (ef) k_decode_scalar<true, true><<<grid, kBlock, 0, s>>>(a);
-        else if (store) k_decode_scalar<false, true><<<grid, kBlock, 0, s>>>(a);
-        else k_decode_scalar<false, false><<<grid, kBlock, 0, s>>>(a);
+        fn = select_decode_scalar(ef, store);
+        grid = shared ? dim3(flat_grid(c, occupancy(c, fn), c->n), 1)
+                      : dim3(per_worker_grid(c, occupancy(c, fn), c->n), c->P);
     }
-    A2_CUDA(cudaGetLastError());
+    A2_CUDA(cudaLaunchKernel(fn, grid, dim3(kBlock), params, 0, s));
+    return A2SGD_OK;
+}
+
+// The single-launch path holds at most kCoopVecPerThread 128-bit vectors of v per thread.
+// Returns the kernel and its grid, or nullptr when (n, P, alignment) does not qualify.
+const void *coop_plan(a2sgd_ctx *c, bool store, bool shared, int vw, uint32_t *grid_out)
+{
+    if (!c->coop_supported || vw < 4) return nullptr;
+    const void *fn = select_coop(!c->alg1, store, shared, c->P);
+    if (!fn) return nullptr;
+    const uint64_t threads = (uint64_t)c->sm_count * occupancy(c, fn) * kBlock;
+    const uint64_t per_thread = kCoopVecPerThread / c->P;
+    const uint64_t n4 = (c->n + 3) / 4;
+    if (n4 > threads * per_thread) return nullptr;
+    const uint64_t need = std::max<uint64_t>(1, (n4 + kBlock - 1) / kBlock);
+    const uint64_t grid = std::min<uint64_t>((uint64_t)c->sm_count * occupancy(c, fn), need);
+    if (grid > c->g_alloc) return nullptr;
+    *grid_out = (uint32_t)grid;
+    return fn;
+}
+
+int launch_coop(a2sgd_ctx *c, const void *fn, uint32_t grid, float *w, int64_t ws, const float *grad, int64_t gs,
+                float *err, int64_t es, float lr, cudaStream_t s)
+{
+    CoopArgs a{};
+    a.enc = make_encode_args(c, grad, gs, err, es, c->local_means, c->pos_counts, nullptr, c->global_means);
+    a.dec = make_decode_args(c, w, ws, grad, gs, err, es, c->local_means, c->global_means, lr);
+    a.barrier = c->barrier;
+    c->coop_epoch += 1;
+    if (c->coop_epoch == 0) c->coop_epoch = 1;
+    a.epoch = c->coop_epoch;
+    const bool never_opens = (c->flags & A2SGD_TEST_BARRIER_NEVER_OPENS) != 0;
+    a.expected = never_opens ? grid + 1 : grid;
+    a.spin_limit = never_opens ? (1u << 12) : (1u << 24); // x 40 ns sleep: ~0.2 ms / ~1 s
+    void *params[] = {&a};
+    A2_CUDA(cudaLaunchCooperativeKernel(fn, dim3(grid), dim3(kBlock), params, 0, s));
     return A2SGD_OK;
 }
 
@@ -211,7 +331,8 @@ extern "C" int a2sgd_create(a2sgd_ctx **out, uint64_t n, uint32_t P, int device,
 {
     if (!out) return A2SGD_ERR_ARG;
     *out = nullptr;
-    const uint32_t known = A2SGD_MODE_ALG1 | A2SGD_FORCE_TWO_PASS | A2SGD_FORCE_COOPERATIVE;
+    const uint32_t known = A2SGD_MODE_ALG1 | A2SGD_FORCE_TWO_PASS | A2SGD_FORCE_COOPERATIVE |
+                           A2SGD_TEST_BARRIER_NEVER_OPENS;
     if (n == 0 || n >= (1ull << 40) || P == 0 || P > (uint32_t)kMaxP || (flags & ~known)) return A2SGD_ERR_ARG;
     if ((flags & A2SGD_FORCE_TWO_PASS) && (flags & A2SGD_FORCE_COOPERATIVE)) return A2SGD_ERR_ARG;
     int count = 0;
@@ -231,19 +352,10 @@ extern "C" int a2sgd_create(a2sgd_ctx **out, uint64_t n, uint32_t P, int device,
         delete c;
         return A2SGD_ERR_CUDA;
     }
-    if (c->alg1) {
-        c->occ_encode = occupancy(k_encode_vec<false, false>);
-        c->occ_decode_repl = occupancy(k_decode_repl_vec<false, true>);
-    } else {
-        c->occ_encode = occupancy(k_encode_vec<true, false>);
-        c->occ_decode_repl = occupancy(k_decode_repl_vec<true, true>);
-    }
-    switch (P) {
-    case 1: c->occ_decode_shared = c->alg1 ? occupancy(k_decode_shared_vec<false, true, 1>) : occupancy(k_decode_shared_vec<true, true, 1>); break;
-    case 2: c->occ_decode_shared = c->alg1 ? occupancy(k_decode_shared_vec<false, true, 2>) : occupancy(k_decode_shared_vec<true, true, 2>); break;
-    case 4: c->occ_decode_shared = c->alg1 ? occupancy(k_decode_shared_vec<false, true, 4>) : occupancy(k_decode_shared_vec<true, true, 4>); break;
-    case 8: c->occ_decode_shared = c->alg1 ? occupancy(k_decode_shared_vec<false, true, 8>) : occupancy(k_decode_shared_vec<true, true, 8>); break;
-    default: c->occ_decode_shared = c->alg1 ? occupancy(k_decode_shared_vec<false, true, 0>) : occupancy(k_decode_shared_vec<true, true, 0>); break;
+    {
+        int coop = 0;
+        if (cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, device) != cudaSuccess) (void)cudaGetLastError();
+        c->coop_supported = coop != 0;
     }
     // partials: room for a (G, P) grid that fills the device at the highest possible occupancy
     const uint32_t max_slots = (uint32_t)c->sm_count * (2048 / kBlock);
@@ -255,6 +367,8 @@ extern "C" int a2sgd_create(a2sgd_ctx **out, uint64_t n, uint32_t P, int device,
     ok = ok && cudaMalloc(&c->pos_counts, sizeof(unsigned long long) * P) == cudaSuccess;
     ok = ok && cudaMalloc(&c->tickets, sizeof(unsigned int) * (P + 1)) == cudaSuccess;
     ok = ok && cudaMalloc(&c->status, sizeof(int)) == cudaSuccess;
+    ok = ok && cudaMalloc(&c->barrier, sizeof(unsigned int) * 2) == cudaSuccess;
+    ok = ok && cudaMemset(c->barrier, 0, sizeof(unsigned int) * 2) == cudaSuccess;
     ok = ok && cudaMemset(c->local_means, 0, sizeof(float) * 2 * P) == cudaSuccess;
     ok = ok && cudaMemset(c->global_means, 0, sizeof(float) * 2) == cudaSuccess;
     ok = ok && cudaMemset(c->pos_counts, 0, sizeof(unsigned long long) * P) == cudaSuccess;
@@ -280,6 +394,7 @@ extern "C" int a2sgd_destroy(a2sgd_ctx *c)
     cudaFree(c->pos_counts);
     cudaFree(c->tickets);
     cudaFree(c->status);
+    cudaFree(c->barrier);
     (void)cudaGetLastError();
     delete c;
     return A2SGD_OK;
@@ -339,15 +454,22 @@ extern "C" int a2sgd_step(a2sgd_ctx *c, float *w, int64_t w_stride, const float 
     if (rc) return rc;
     if (w_stride != 0 && !stride_ok(w_stride, c->n, c->P)) return A2SGD_ERR_ARG;
     if (!aligned(w, 4)) return A2SGD_ERR_ALIGN;
-    if (c->flags & A2SGD_FORCE_COOPERATIVE) return A2SGD_ERR_TOO_LARGE;
     DeviceGuard guard(c->device);
     if (!guard.ok) return A2SGD_ERR_CUDA;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const int64_t ws = (c->P == 1) ? 0 : w_stride;
+    if (!(c->flags & A2SGD_FORCE_TWO_PASS)) {
+        const bool store = !c->alg1 || err != nullptr;
+        const int vw = decode_vec_width(c, w, ws, grad, grad_stride, err, err_stride);
+        uint32_t grid = 0;
+        const void *fn = coop_plan(c, store, ws == 0, vw, &grid);
+        if (fn) return launch_coop(c, fn, grid, w, ws, grad, grad_stride, err, err_stride, lr, s);
+        if (c->flags & A2SGD_FORCE_COOPERATIVE) return A2SGD_ERR_TOO_LARGE;
+    }
     const int r1 = launch_encode(c, grad, grad_stride, err, err_stride, c->local_means, c->pos_counts, nullptr,
                                  c->global_means, s);
     if (r1) return r1;
-    return launch_decode(c, w, (c->P == 1) ? 0 : w_stride, grad, grad_stride, err, err_stride, c->local_means,
-                         c->global_means, lr, s);
+    return launch_decode(c, w, ws, grad, grad_stride, err, err_stride, c->local_means, c->global_means, lr, s);
 }
 
 extern "C" int a2sgd_step_host(a2sgd_ctx *c, float *w, int64_t w_stride, const float *grad_host,
@@ -393,6 +515,11 @@ extern "C" int a2sgd_read_stats(a2sgd_ctx *c, float *local_means_host, float *gl
     A2_CUDA(cudaMemcpyAsync(&st, c->status, sizeof(int), cudaMemcpyDeviceToHost, s));
     A2_CUDA(cudaMemsetAsync(c->status, 0, sizeof(int), s));
     A2_CUDA(cudaStreamSynchronize(s));
+    if (st == A2SGD_ERR_TIMEOUT) {
+        // CTAs that gave up left their arrivals in the barrier counter
+        A2_CUDA(cudaMemsetAsync(c->barrier, 0, sizeof(unsigned int), s));
+        A2_CUDA(cudaStreamSynchronize(s));
+    }
     if (device_status) *device_status = st;
     return A2SGD_OK;
 }
@@ -400,12 +527,25 @@ extern "C" int a2sgd_read_stats(a2sgd_ctx *c, float *local_means_host, float *gl
 extern "C" int a2sgd_launch_info(a2sgd_ctx *c, int64_t w_stride, uint32_t out[5])
 {
     if (!c || !out) return A2SGD_ERR_ARG;
-    const uint64_t items = (c->n + 3) / 4;
-    out[0] = per_worker_grid(c, c->occ_encode, items) * c->P;
-    out[1] = (w_stride == 0 || c->P == 1) ? flat_grid(c, c->occ_decode_shared, items)
-                                          : per_worker_grid(c, c->occ_decode_repl, items) * c->P;
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return A2SGD_ERR_CUDA;
+    // geometry for best-aligned buffers (what a caller that pads rows to 128 bytes gets)
+    const bool ef = !c->alg1;
+    const bool shared = w_stride == 0 || c->P == 1;
+    const int vw = A2SGD_MAX_VW >= 8 ? 8 : 4;
+    const uint64_t items = (c->n + vw - 1) / vw;
+    out[0] = per_worker_grid(c, occupancy(c, select_encode(ef, false, vw)), items) * c->P;
+    out[1] = shared ? flat_grid(c, occupancy(c, select_decode_shared(ef, true, c->P, vw)), items)
+                    : per_worker_grid(c, occupancy(c, select_decode_repl(ef, true, vw)), items) * c->P;
     out[2] = kBlock;
     out[3] = 0;
+    if (!(c->flags & A2SGD_FORCE_TWO_PASS)) {
+        uint32_t grid = 0;
+        if (coop_plan(c, true, shared, vw, &grid)) {
+            out[3] = 1;
+            out[0] = out[1] = grid;
+        }
+    }
     out[4] = (uint32_t)c->sm_count;
     return A2SGD_OK;
 }

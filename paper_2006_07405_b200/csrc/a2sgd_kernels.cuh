@@ -44,28 +44,59 @@ struct __align__(8) Partial {
 };
 
 // ------------------------------------------------------------------ memory access helpers
-// Streaming 128-bit accesses.  Every byte on this path is touched at most
-// twice per step (once by K1, once by K3) with gigabytes in between, so L1
-// allocation is pointless and L2 lines should be first in line for eviction.
-__device__ __forceinline__ float4 ld_stream(const float *p)
+// Streaming vector accesses, VW = 4 (128-bit) or 8 (256-bit, new on sm_100).
+// Every byte on this path is touched at most twice per step (once by K1, once
+// by K3) with gigabytes in between, so nothing is allocated in L1; the 256-bit
+// forms also mark their L2 lines evict-first (the ISA ties that hint to the
+// 256-bit width).
+template <int VW>
+struct Vec {
+    float v[VW];
+};
+
+template <int VW>
+__device__ __forceinline__ Vec<VW> ld_vec(const float *p);
+template <>
+__device__ __forceinline__ Vec<4> ld_vec<4>(const float *p)
 {
-    float4 r;
+    Vec<4> r;
     asm volatile("ld.global.L1::no_allocate.v4.f32 {%0,%1,%2,%3}, [%4];"
-                 : "=f"(r.x), "=f"(r.y), "=f"(r.z), "=f"(r.w)
+                 : "=f"(r.v[0]), "=f"(r.v[1]), "=f"(r.v[2]), "=f"(r.v[3])
                  : "l"(p));
     return r;
+}
+template <>
+__device__ __forceinline__ Vec<8> ld_vec<8>(const float *p)
+{
+    Vec<8> r;
+    asm volatile("ld.global.L1::no_allocate.L2::evict_first.v8.f32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                 : "=f"(r.v[0]), "=f"(r.v[1]), "=f"(r.v[2]), "=f"(r.v[3]), "=f"(r.v[4]), "=f"(r.v[5]),
+                   "=f"(r.v[6]), "=f"(r.v[7])
+                 : "l"(p));
+    return r;
+}
+template <int VW>
+__device__ __forceinline__ void st_vec(float *p, const Vec<VW> &x);
+template <>
+__device__ __forceinline__ void st_vec<4>(float *p, const Vec<4> &x)
+{
+    asm volatile("st.global.L1::no_allocate.v4.f32 [%0], {%1,%2,%3,%4};" ::"l"(p), "f"(x.v[0]), "f"(x.v[1]),
+                 "f"(x.v[2]), "f"(x.v[3])
+                 : "memory");
+}
+template <>
+__device__ __forceinline__ void st_vec<8>(float *p, const Vec<8> &x)
+{
+    asm volatile("st.global.L1::no_allocate.L2::evict_first.v8.f32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(p),
+                 "f"(x.v[0]), "f"(x.v[1]), "f"(x.v[2]), "f"(x.v[3]), "f"(x.v[4]), "f"(x.v[5]), "f"(x.v[6]),
+                 "f"(x.v[7])
+                 : "memory");
 }
 __device__ __forceinline__ float ld_stream1(const float *p)
 {
     float r;
     asm volatile("ld.global.L1::no_allocate.f32 %0, [%1];" : "=f"(r) : "l"(p));
     return r;
-}
-__device__ __forceinline__ void st_stream(float *p, float4 v)
-{
-    asm volatile("st.global.L1::no_allocate.v4.f32 [%0], {%1,%2,%3,%4};" ::"l"(p),
-                 "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w)
-                 : "memory");
 }
 __device__ __forceinline__ void st_stream1(float *p, float v)
 {
@@ -91,23 +122,37 @@ __device__ __forceinline__ void split1(float v, float &sp, float &sn, unsigned &
     bit = p ? 1u : 0u;
 }
 
-// One 4-vector: pairwise fp32 sums of the two groups, count, 4-bit pos nibble.
-__device__ __forceinline__ void split4(float4 v, float &sp, float &sn, unsigned &c, unsigned &nib)
+// Pairwise fp32 sum of VW values (VW a power of two).
+template <int VW>
+__device__ __forceinline__ float tree_sum(const float *x)
 {
-    float p0, p1, p2, p3, n0, n1, n2, n3;
-    unsigned b0, b1, b2, b3;
-    split1(v.x, p0, n0, c, b0);
-    split1(v.y, p1, n1, c, b1);
-    split1(v.z, p2, n2, c, b2);
-    split1(v.w, p3, n3, c, b3);
-    sp = (p0 + p1) + (p2 + p3);
-    sn = (n0 + n1) + (n2 + n3);
-    nib = b0 | (b1 << 1) | (b2 << 2) | (b3 << 3);
+    if (VW == 1) return x[0];
+    return tree_sum<(VW > 1 ? VW / 2 : 1)>(x) + tree_sum<(VW > 1 ? VW / 2 : 1)>(x + VW / 2);
 }
 
-__device__ __forceinline__ float4 add4(float4 a, float4 b)
+// One vector: pairwise fp32 sums of the two groups, count, VW-bit pos field.
+template <int VW>
+__device__ __forceinline__ void split_vec(const Vec<VW> &v, float &sp, float &sn, unsigned &c, unsigned &bits)
 {
-    return make_float4(a.x + b.x, a.y + b.y, a.z + b.z, a.w + b.w);
+    float ps[VW], ns[VW];
+    bits = 0;
+#pragma unroll
+    for (int k = 0; k < VW; ++k) {
+        unsigned b;
+        split1(v.v[k], ps[k], ns[k], c, b);
+        bits |= b << k;
+    }
+    sp = tree_sum<VW>(ps);
+    sn = tree_sum<VW>(ns);
+}
+
+template <int VW>
+__device__ __forceinline__ Vec<VW> add_vec(const Vec<VW> &a, const Vec<VW> &b)
+{
+    Vec<VW> r;
+#pragma unroll
+    for (int k = 0; k < VW; ++k) r.v[k] = a.v[k] + b.v[k];
+    return r;
 }
 
 // ------------------------------------------------------------------ fixed-order block reduction
@@ -231,13 +276,16 @@ __device__ __forceinline__ void finish_worker(const EncodeArgs &a, uint32_t p, d
     }
 }
 
-// Fast path: 16-byte aligned bases, strides multiple of 4.  grid = (G, P).
-// Lanes are handled in groups of 8 (= one 32-element mask word) whose loop
-// bounds are uniform across the group, so the sub-warp shuffles that assemble
-// a mask word always see all eight lanes.
-template <bool EF, bool MASK>
+// Fast path, VW floats per access: bases aligned to 4*VW bytes, worker strides
+// multiples of VW elements.  grid = (G, P).  Lanes are handled in groups of
+// 32/VW (= one 32-element mask word) whose loop bounds are uniform across the
+// group, so the sub-warp shuffles that assemble a mask word always see the
+// whole group.
+template <bool EF, bool MASK, int VW>
 __global__ void __launch_bounds__(kBlock) k_encode_vec(EncodeArgs a)
 {
+    constexpr int LPW = 32 / VW;  // lanes per mask word
+    constexpr int U = 16 / VW;    // vectors per trip: 16 elements per thread per batch
     __shared__ double sh_d[2][kWarps];
     __shared__ unsigned long long sh_n[kWarps];
     __shared__ int sh_flag;
@@ -245,67 +293,66 @@ __global__ void __launch_bounds__(kBlock) k_encode_vec(EncodeArgs a)
     const uint32_t p = blockIdx.y;
     const float *__restrict__ g = a.grad + (int64_t)p * a.grad_stride;
     const float *__restrict__ e = EF ? a.err + (int64_t)p * a.err_stride : nullptr;
-    const uint64_t n4 = a.n >> 2;
+    const uint64_t nv = a.n / VW;
     const uint64_t full_words = a.n >> 5;
     uint32_t *mask = MASK ? a.pos_mask + (uint64_t)p * ((a.n + 31) >> 5) : nullptr;
 
     const unsigned lane = threadIdx.x & 31u;
-    const unsigned sub = lane & 7u;
-    const unsigned group_mask = 0xffu << (lane & ~7u);
+    const unsigned sub = lane & (LPW - 1);
+    const unsigned group_mask = ((1u << LPW) - 1u) << (lane & ~(unsigned)(LPW - 1));
     const uint64_t stride = (uint64_t)gridDim.x * kBlock;
     uint64_t j = (uint64_t)blockIdx.x * kBlock + threadIdx.x;
 
     Acc acc;
 
-    auto emit_word = [&](unsigned nib, uint64_t jv) {
+    auto emit_word = [&](unsigned bits, uint64_t jv) {
         if (MASK) {
-            unsigned w = nib << (4u * sub);
-            w |= __shfl_xor_sync(group_mask, w, 1);
-            w |= __shfl_xor_sync(group_mask, w, 2);
-            w |= __shfl_xor_sync(group_mask, w, 4);
-            const uint64_t word = jv >> 3;
+            unsigned w = bits << (VW * sub);
+#pragma unroll
+            for (int x = 1; x < LPW; x <<= 1) w |= __shfl_xor_sync(group_mask, w, x);
+            const uint64_t word = jv / LPW;
             if (sub == 0 && word < full_words) mask[word] = w;
         }
     };
 
-    // main loop: 4 vectors per thread per trip, all loads issued before use
-    for (; (j - sub + 7) + 3 * stride < n4; j += 4 * stride) {
-        float4 gv[4], ev[4];
+    // main loop: U vectors per thread per trip, all loads issued before use
+    for (; (j - sub + (LPW - 1)) + (U - 1) * stride < nv; j += U * stride) {
+        Vec<VW> gv[U], ev[U];
 #pragma unroll
-        for (int u = 0; u < 4; ++u) gv[u] = ld_stream(g + 4 * (j + u * stride));
+        for (int u = 0; u < U; ++u) gv[u] = ld_vec<VW>(g + VW * (j + u * stride));
         if (EF) {
 #pragma unroll
-            for (int u = 0; u < 4; ++u) ev[u] = ld_stream(e + 4 * (j + u * stride));
+            for (int u = 0; u < U; ++u) ev[u] = ld_vec<VW>(e + VW * (j + u * stride));
         }
-        float sp[4], sn[4];
-        unsigned nib[4];
+        float sp[U], sn[U];
+        unsigned bits[U];
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
-            const float4 v = EF ? add4(gv[u], ev[u]) : gv[u];
-            split4(v, sp[u], sn[u], acc.n_pos, nib[u]);
+        for (int u = 0; u < U; ++u) {
+            const Vec<VW> v = EF ? add_vec<VW>(gv[u], ev[u]) : gv[u];
+            split_vec<VW>(v, sp[u], sn[u], acc.n_pos, bits[u]);
         }
-        acc.s_pos += (double)((sp[0] + sp[1]) + (sp[2] + sp[3]));
-        acc.s_neg += (double)((sn[0] + sn[1]) + (sn[2] + sn[3]));
+        acc.s_pos += (double)tree_sum<U>(sp);
+        acc.s_neg += (double)tree_sum<U>(sn);
 #pragma unroll
-        for (int u = 0; u < 4; ++u) emit_word(nib[u], j + u * stride);
+        for (int u = 0; u < U; ++u) emit_word(bits[u], j + u * stride);
     }
-    // remainder: one vector per trip, bounds uniform per group of 8 lanes
-    for (; (j - sub) < n4; j += stride) {
+    // remainder: one vector per trip, bounds uniform per lane group
+    for (; (j - sub) < nv; j += stride) {
         float sp = 0.f, sn = 0.f;
-        unsigned nib = 0;
-        if (j < n4) {
-            float4 v = ld_stream(g + 4 * j);
-            if (EF) v = add4(v, ld_stream(e + 4 * j));
-            split4(v, sp, sn, acc.n_pos, nib);
+        unsigned bits = 0;
+        if (j < nv) {
+            Vec<VW> v = ld_vec<VW>(g + VW * j);
+            if (EF) v = add_vec<VW>(v, ld_vec<VW>(e + VW * j));
+            split_vec<VW>(v, sp, sn, acc.n_pos, bits);
         }
         acc.s_pos += (double)sp;
         acc.s_neg += (double)sn;
-        emit_word(nib, j);
+        emit_word(bits, j);
     }
     if (blockIdx.x == 0) {
-        // the n % 4 trailing elements
-        const uint64_t i = (n4 << 2) + threadIdx.x;
-        if (threadIdx.x < 4 && i < a.n) {
+        // the n % VW trailing elements
+        const uint64_t i = nv * VW + threadIdx.x;
+        if (threadIdx.x < VW && i < a.n) {
             float v = ld_stream1(g + i);
             if (EF) v += ld_stream1(e + i);
             float sp, sn;
@@ -445,75 +492,90 @@ __device__ __forceinline__ void decode1(float v, const WorkerConst &c, float &g_
     }
 }
 
-template <bool EF>
-__device__ __forceinline__ void decode4(float4 v, const WorkerConst &c, float4 &g_hat, float4 &resid)
+template <bool EF, int VW>
+__device__ __forceinline__ void decode_vec(const Vec<VW> &v, const WorkerConst &c, Vec<VW> &g_hat, Vec<VW> &resid)
 {
-    decode1<EF>(v.x, c, g_hat.x, resid.x);
-    decode1<EF>(v.y, c, g_hat.y, resid.y);
-    decode1<EF>(v.z, c, g_hat.z, resid.z);
-    decode1<EF>(v.w, c, g_hat.w, resid.w);
+#pragma unroll
+    for (int k = 0; k < VW; ++k) decode1<EF>(v.v[k], c, g_hat.v[k], resid.v[k]);
 }
 
-// One shared w: each thread owns a 4-vector of the model and walks the P
+template <int VW>
+__device__ __forceinline__ Vec<VW> axpy_vec(float alpha, const Vec<VW> &x, const Vec<VW> &y)
+{
+    Vec<VW> r;
+#pragma unroll
+    for (int k = 0; k < VW; ++k) r.v[k] = fmaf(alpha, x.v[k], y.v[k]);
+    return r;
+}
+
+template <int VW>
+__device__ __forceinline__ Vec<VW> zero_vec()
+{
+    Vec<VW> r;
+#pragma unroll
+    for (int k = 0; k < VW; ++k) r.v[k] = 0.f;
+    return r;
+}
+
+// One shared w: each thread owns a VW-vector of the model and walks the P
 // workers in order (fixed summation order), so w is read and written once
 // per model element.  PT > 0: P known at compile time (all 2P+1 loads of a
 // vector are issued before any is used); PT == 0: run-time P.
-template <bool EF, bool STORE, int PT>
+template <bool EF, bool STORE, int PT, int VW>
 __global__ void __launch_bounds__(kBlock) k_decode_shared_vec(DecodeArgs a)
 {
     __shared__ WorkerConst sh_c[PT > 0 ? 1 : kMaxP];
     const uint32_t P = PT > 0 ? PT : a.P;
     const float m_pos = __ldg(a.global_means), m_neg = __ldg(a.global_means + 1);
     const float scale = -a.lr / (float)P;
-    const uint64_t n4 = a.n >> 2;
+    const uint64_t nv = a.n / VW;
     const uint64_t stride = (uint64_t)gridDim.x * kBlock;
 
     if (PT > 0) {
-        WorkerConst c[PT > 0 ? PT : 1];
+        constexpr int PP = PT > 0 ? PT : 1;
+        WorkerConst c[PP];
 #pragma unroll
-        for (int p = 0; p < PT; ++p) c[p] = worker_const<EF>(a, p, m_pos, m_neg);
-        for (uint64_t j = (uint64_t)blockIdx.x * kBlock + threadIdx.x; j < n4; j += stride) {
-            float4 gv[PT > 0 ? PT : 1], ev[PT > 0 ? PT : 1];
-            const float4 wv = ld_stream(a.w + 4 * j);
+        for (int p = 0; p < PP; ++p) c[p] = worker_const<EF>(a, p, m_pos, m_neg);
+        for (uint64_t j = (uint64_t)blockIdx.x * kBlock + threadIdx.x; j < nv; j += stride) {
+            Vec<VW> gv[PP], ev[PP];
+            const Vec<VW> wv = ld_vec<VW>(a.w + VW * j);
 #pragma unroll
-            for (int p = 0; p < PT; ++p) gv[p] = ld_stream(a.grad + (int64_t)p * a.grad_stride + 4 * j);
+            for (int p = 0; p < PP; ++p) gv[p] = ld_vec<VW>(a.grad + (int64_t)p * a.grad_stride + VW * j);
             if (EF) {
 #pragma unroll
-                for (int p = 0; p < PT; ++p) ev[p] = ld_stream(a.err + (int64_t)p * a.err_stride + 4 * j);
+                for (int p = 0; p < PP; ++p) ev[p] = ld_vec<VW>(a.err + (int64_t)p * a.err_stride + VW * j);
             }
-            float4 sum = make_float4(0.f, 0.f, 0.f, 0.f);
+            Vec<VW> sum = zero_vec<VW>();
 #pragma unroll
-            for (int p = 0; p < PT; ++p) {
-                const float4 v = EF ? add4(gv[p], ev[p]) : gv[p];
-                float4 gh, rs;
-                decode4<EF>(v, c[p], gh, rs);
-                sum = add4(sum, gh);
-                if (STORE) st_stream(a.err + (int64_t)p * a.err_stride + 4 * j, rs);
+            for (int p = 0; p < PP; ++p) {
+                const Vec<VW> v = EF ? add_vec<VW>(gv[p], ev[p]) : gv[p];
+                Vec<VW> gh, rs;
+                decode_vec<EF, VW>(v, c[p], gh, rs);
+                sum = add_vec<VW>(sum, gh);
+                if (STORE) st_vec<VW>(a.err + (int64_t)p * a.err_stride + VW * j, rs);
             }
-            st_stream(a.w + 4 * j, make_float4(fmaf(scale, sum.x, wv.x), fmaf(scale, sum.y, wv.y),
-                                               fmaf(scale, sum.z, wv.z), fmaf(scale, sum.w, wv.w)));
+            st_vec<VW>(a.w + VW * j, axpy_vec<VW>(scale, sum, wv));
         }
     } else {
         for (uint32_t p = threadIdx.x; p < P; p += kBlock) sh_c[p] = worker_const<EF>(a, p, m_pos, m_neg);
         __syncthreads();
-        for (uint64_t j = (uint64_t)blockIdx.x * kBlock + threadIdx.x; j < n4; j += stride) {
-            const float4 wv = ld_stream(a.w + 4 * j);
-            float4 sum = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (uint64_t j = (uint64_t)blockIdx.x * kBlock + threadIdx.x; j < nv; j += stride) {
+            const Vec<VW> wv = ld_vec<VW>(a.w + VW * j);
+            Vec<VW> sum = zero_vec<VW>();
             for (uint32_t p = 0; p < P; ++p) {
-                float4 v = ld_stream(a.grad + (int64_t)p * a.grad_stride + 4 * j);
-                if (EF) v = add4(v, ld_stream(a.err + (int64_t)p * a.err_stride + 4 * j));
-                float4 gh, rs;
-                decode4<EF>(v, sh_c[p], gh, rs);
-                sum = add4(sum, gh);
-                if (STORE) st_stream(a.err + (int64_t)p * a.err_stride + 4 * j, rs);
+                Vec<VW> v = ld_vec<VW>(a.grad + (int64_t)p * a.grad_stride + VW * j);
+                if (EF) v = add_vec<VW>(v, ld_vec<VW>(a.err + (int64_t)p * a.err_stride + VW * j));
+                Vec<VW> gh, rs;
+                decode_vec<EF, VW>(v, sh_c[p], gh, rs);
+                sum = add_vec<VW>(sum, gh);
+                if (STORE) st_vec<VW>(a.err + (int64_t)p * a.err_stride + VW * j, rs);
             }
-            st_stream(a.w + 4 * j, make_float4(fmaf(scale, sum.x, wv.x), fmaf(scale, sum.y, wv.y),
-                                               fmaf(scale, sum.z, wv.z), fmaf(scale, sum.w, wv.w)));
+            st_vec<VW>(a.w + VW * j, axpy_vec<VW>(scale, sum, wv));
         }
     }
-    // the n % 4 trailing elements
-    if (blockIdx.x == 0 && threadIdx.x < 4) {
-        const uint64_t i = (n4 << 2) + threadIdx.x;
+    // the n % VW trailing elements
+    if (blockIdx.x == 0 && threadIdx.x < VW) {
+        const uint64_t i = nv * VW + threadIdx.x;
         if (i < a.n) {
             float sum = 0.f;
             for (uint32_t p = 0; p < P; ++p) {
@@ -531,7 +593,7 @@ __global__ void __launch_bounds__(kBlock) k_decode_shared_vec(DecodeArgs a)
 }
 
 // One w replica per worker (Algorithm 1's layout).  grid = (G, P).
-template <bool EF, bool STORE>
+template <bool EF, bool STORE, int VW>
 __global__ void __launch_bounds__(kBlock) k_decode_repl_vec(DecodeArgs a)
 {
     const uint32_t p = blockIdx.y;
@@ -541,43 +603,40 @@ __global__ void __launch_bounds__(kBlock) k_decode_repl_vec(DecodeArgs a)
     float *e = (EF || STORE) ? a.err + (int64_t)p * a.err_stride : nullptr;
     float *w = a.w + (int64_t)p * a.w_stride;
     const float neg_lr = -a.lr;
-    const uint64_t n4 = a.n >> 2;
+    const uint64_t nv = a.n / VW;
     const uint64_t stride = (uint64_t)gridDim.x * kBlock;
     uint64_t j = (uint64_t)blockIdx.x * kBlock + threadIdx.x;
-    constexpr int U = 2;
-    for (; j + (U - 1) * stride < n4; j += U * stride) {
-        float4 gv[U], ev[U], wv[U];
+    constexpr int U = 8 / VW;
+    for (; j + (U - 1) * stride < nv; j += U * stride) {
+        Vec<VW> gv[U], ev[U], wv[U];
 #pragma unroll
-        for (int u = 0; u < U; ++u) gv[u] = ld_stream(g + 4 * (j + u * stride));
+        for (int u = 0; u < U; ++u) gv[u] = ld_vec<VW>(g + VW * (j + u * stride));
         if (EF) {
 #pragma unroll
-            for (int u = 0; u < U; ++u) ev[u] = ld_stream(e + 4 * (j + u * stride));
+            for (int u = 0; u < U; ++u) ev[u] = ld_vec<VW>(e + VW * (j + u * stride));
         }
 #pragma unroll
-        for (int u = 0; u < U; ++u) wv[u] = ld_stream(w + 4 * (j + u * stride));
+        for (int u = 0; u < U; ++u) wv[u] = ld_vec<VW>(w + VW * (j + u * stride));
 #pragma unroll
         for (int u = 0; u < U; ++u) {
-            const float4 v = EF ? add4(gv[u], ev[u]) : gv[u];
-            float4 gh, rs;
-            decode4<EF>(v, c, gh, rs);
-            if (STORE) st_stream(e + 4 * (j + u * stride), rs);
-            st_stream(w + 4 * (j + u * stride),
-                      make_float4(fmaf(neg_lr, gh.x, wv[u].x), fmaf(neg_lr, gh.y, wv[u].y),
-                                  fmaf(neg_lr, gh.z, wv[u].z), fmaf(neg_lr, gh.w, wv[u].w)));
+            const Vec<VW> v = EF ? add_vec<VW>(gv[u], ev[u]) : gv[u];
+            Vec<VW> gh, rs;
+            decode_vec<EF, VW>(v, c, gh, rs);
+            if (STORE) st_vec<VW>(e + VW * (j + u * stride), rs);
+            st_vec<VW>(w + VW * (j + u * stride), axpy_vec<VW>(neg_lr, gh, wv[u]));
         }
     }
-    for (; j < n4; j += stride) {
-        float4 v = ld_stream(g + 4 * j);
-        if (EF) v = add4(v, ld_stream(e + 4 * j));
-        const float4 wv = ld_stream(w + 4 * j);
-        float4 gh, rs;
-        decode4<EF>(v, c, gh, rs);
-        if (STORE) st_stream(e + 4 * j, rs);
-        st_stream(w + 4 * j, make_float4(fmaf(neg_lr, gh.x, wv.x), fmaf(neg_lr, gh.y, wv.y),
-                                         fmaf(neg_lr, gh.z, wv.z), fmaf(neg_lr, gh.w, wv.w)));
+    for (; j < nv; j += stride) {
+        Vec<VW> v = ld_vec<VW>(g + VW * j);
+        if (EF) v = add_vec<VW>(v, ld_vec<VW>(e + VW * j));
+        const Vec<VW> wv = ld_vec<VW>(w + VW * j);
+        Vec<VW> gh, rs;
+        decode_vec<EF, VW>(v, c, gh, rs);
+        if (STORE) st_vec<VW>(e + VW * j, rs);
+        st_vec<VW>(w + VW * j, axpy_vec<VW>(neg_lr, gh, wv));
     }
-    if (blockIdx.x == 0 && threadIdx.x < 4) {
-        const uint64_t i = (n4 << 2) + threadIdx.x;
+    if (blockIdx.x == 0 && threadIdx.x < VW) {
+        const uint64_t i = nv * VW + threadIdx.x;
         if (i < a.n) {
             float v = ld_stream1(g + i);
             if (EF) v += ld_stream1(e + i);
@@ -612,6 +671,229 @@ __global__ void __launch_bounds__(kBlock) k_decode_scalar(DecodeArgs a)
         }
         float *wp = a.w + (int64_t)p_lo * a.w_stride + i;
         *wp = fmaf(scale, sum, *wp);
+    }
+}
+
+// ------------------------------------------------------------------ K4: single cooperative launch
+// For n*P small enough that every thread can keep its share of v in
+// registers: phase 1 loads g (and e) once and reduces, a grid-wide barrier
+// publishes the means, phase 2 decodes from the registers.  HBM traffic is
+// 20 B per worker-element instead of 28, and one launch instead of two.
+// Must be launched cooperatively (all CTAs co-resident).  The barrier wait is
+// bounded: a CTA that gives up latches kDevTimeout and returns without
+// writing any output.
+struct CoopArgs {
+    EncodeArgs enc;            // pos_mask unused; global_means required
+    DecodeArgs dec;
+    unsigned int *barrier;     // [0] arrival counter (zero between launches), [1] release epoch
+    unsigned int epoch;        // value that opens the barrier for this launch (never 0)
+    unsigned int expected;     // arrivals that open the barrier (= gridDim.x in normal use)
+    unsigned int spin_limit;   // polls before giving up
+};
+
+constexpr int kCoopVecPerThread = 8; // 128-bit vectors of v a thread may hold, summed over its workers
+
+__device__ __forceinline__ unsigned int ld_acquire_u32(const unsigned int *p)
+{
+    unsigned int v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void st_release_u32(unsigned int *p, unsigned int v)
+{
+    asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+
+template <bool EF, bool STORE, int PT, bool SHARED>
+__global__ void __launch_bounds__(kBlock) k_step_coop(CoopArgs a)
+{
+    constexpr int K = kCoopVecPerThread / PT;
+    __shared__ double sh_d[2][kWarps];
+    __shared__ unsigned long long sh_n[kWarps];
+    __shared__ int sh_flag;
+
+    const EncodeArgs &ea = a.enc;
+    const DecodeArgs &da = a.dec;
+    const uint64_t n4 = ea.n >> 2;
+    const uint64_t T = (uint64_t)gridDim.x * kBlock;
+    const uint64_t tid = (uint64_t)blockIdx.x * kBlock + threadIdx.x;
+    const bool has_tail = blockIdx.x == 0 && threadIdx.x < 4 && (n4 << 2) + threadIdx.x < ea.n;
+    const uint64_t i_tail = (n4 << 2) + threadIdx.x;
+
+    // ---- phase 1: load, form v, reduce per worker
+    Vec<4> v[PT][K];
+    float v_tail[PT];
+    Acc acc[PT];
+#pragma unroll
+    for (int p = 0; p < PT; ++p) {
+        const float *g = ea.grad + (int64_t)p * ea.grad_stride;
+        const float *e = EF ? ea.err + (int64_t)p * ea.err_stride : nullptr;
+#pragma unroll
+        for (int k = 0; k < K; ++k) {
+            const uint64_t j = tid + (uint64_t)k * T;
+            v[p][k] = zero_vec<4>();
+            if (j < n4) {
+                v[p][k] = ld_vec<4>(g + 4 * j);
+                if (EF) v[p][k] = add_vec<4>(v[p][k], ld_vec<4>(e + 4 * j));
+            }
+        }
+        v_tail[p] = 0.f;
+        if (has_tail) {
+            v_tail[p] = ld_stream1(g + i_tail);
+            if (EF) v_tail[p] += ld_stream1(e + i_tail);
+        }
+    }
+#pragma unroll
+    for (int p = 0; p < PT; ++p) {
+        float sp[K], sn[K];
+#pragma unroll
+        for (int k = 0; k < K; ++k) {
+            sp[k] = sn[k] = 0.f;
+            unsigned bits;
+            if (tid + (uint64_t)k * T < n4) split_vec<4>(v[p][k], sp[k], sn[k], acc[p].n_pos, bits);
+        }
+        acc[p].s_pos = (double)tree_sum<K>(sp);
+        acc[p].s_neg = (double)tree_sum<K>(sn);
+        if (has_tail) {
+            float tp, tn;
+            unsigned bit;
+            split1(v_tail[p], tp, tn, acc[p].n_pos, bit);
+            acc[p].s_pos += (double)tp;
+            acc[p].s_neg += (double)tn;
+        }
+    }
+    const uint32_t G = gridDim.x;
+#pragma unroll
+    for (int p = 0; p < PT; ++p) {
+        double s_pos = acc[p].s_pos, s_neg = acc[p].s_neg;
+        unsigned long long n_pos = acc[p].n_pos;
+        block_reduce(s_pos, s_neg, n_pos, sh_d, sh_n);
+        if (threadIdx.x == 0) {
+            Partial *mine = ea.partials + (uint64_t)p * G;
+            mine[blockIdx.x].s_pos = s_pos;
+            mine[blockIdx.x].s_neg = s_neg;
+            mine[blockIdx.x].n_pos = n_pos;
+        }
+    }
+    // ---- grid barrier: the last CTA to arrive folds the partials and opens it
+    if (threadIdx.x == 0) {
+        __threadfence();
+        const unsigned int t = atomicAdd(&a.barrier[0], 1u);
+        sh_flag = (t == a.expected - 1) ? 1 : 0;
+    }
+    __syncthreads();
+    if (sh_flag) {
+        __threadfence();
+        for (uint32_t p = 0; p < PT; ++p) {
+            const Partial *part = ea.partials + (uint64_t)p * G;
+            double fp = 0.0, fn = 0.0;
+            unsigned long long fc = 0;
+            for (uint32_t i = threadIdx.x; i < G; i += kBlock) {
+                fp += __ldcg(&part[i].s_pos);
+                fn += __ldcg(&part[i].s_neg);
+                fc += __ldcg(&part[i].n_pos);
+            }
+            __syncthreads();
+            block_reduce(fp, fn, fc, sh_d, sh_n);
+            if (threadIdx.x == 0) {
+                const unsigned long long n_neg = ea.n - fc;
+                ea.local_means[2 * p + 0] = fc ? (float)(fp / (double)fc) : 0.0f;
+                ea.local_means[2 * p + 1] = n_neg ? (float)(fn / (double)n_neg) : 0.0f;
+                if (ea.pos_counts) ea.pos_counts[p] = fc;
+                if (!isfinite(fp) || !isfinite(fn)) atomicCAS(ea.status, kDevOk, kDevNonFinite);
+            }
+        }
+        if (threadIdx.x == 0) {
+            double gp = 0.0, gn = 0.0;
+            for (uint32_t q = 0; q < PT; ++q) { // worker order
+                gp += (double)ea.local_means[2 * q + 0];
+                gn += (double)ea.local_means[2 * q + 1];
+            }
+            ea.global_means[0] = (float)(gp / (double)PT);
+            ea.global_means[1] = (float)(gn / (double)PT);
+            a.barrier[0] = 0;
+            __threadfence();
+            st_release_u32(&a.barrier[1], a.epoch);
+        }
+        __syncthreads();
+    } else {
+        if (threadIdx.x == 0) {
+            unsigned int polls = 0;
+            int ok = 1;
+            while (ld_acquire_u32(&a.barrier[1]) != a.epoch) {
+                if (++polls > a.spin_limit) {
+                    ok = 0;
+                    break;
+                }
+                __nanosleep(40);
+            }
+            if (!ok) atomicCAS(ea.status, kDevOk, kDevTimeout);
+            sh_flag = ok ? 2 : -1;
+        }
+        __syncthreads();
+        if (sh_flag < 0) return; // gave up: no output is written by this CTA
+    }
+    // ---- phase 2: decode from registers
+    const float m_pos = __ldcg(ea.global_means), m_neg = __ldcg(ea.global_means + 1);
+    WorkerConst c[PT];
+#pragma unroll
+    for (int p = 0; p < PT; ++p) {
+        if (EF) {
+            c[p].a_pos = m_pos;
+            c[p].a_neg = -m_neg;
+            c[p].b_pos = c[p].b_neg = 0.f;
+        } else {
+            const float mu_pos = __ldcg(ea.local_means + 2 * p), mu_neg = __ldcg(ea.local_means + 2 * p + 1);
+            c[p].a_pos = m_pos - mu_pos;
+            c[p].a_neg = mu_neg - m_neg;
+            c[p].b_pos = mu_pos;
+            c[p].b_neg = -mu_neg;
+        }
+    }
+    const float scale = SHARED ? -da.lr / (float)PT : -da.lr;
+#pragma unroll
+    for (int k = 0; k < K; ++k) {
+        const uint64_t j = tid + (uint64_t)k * T;
+        if (j >= n4) continue;
+        if (SHARED) {
+            const Vec<4> wv = ld_vec<4>(da.w + 4 * j);
+            Vec<4> sum = zero_vec<4>();
+#pragma unroll
+            for (int p = 0; p < PT; ++p) {
+                Vec<4> gh, rs;
+                decode_vec<EF, 4>(v[p][k], c[p], gh, rs);
+                sum = add_vec<4>(sum, gh);
+                if (STORE) st_vec<4>(da.err + (int64_t)p * da.err_stride + 4 * j, rs);
+            }
+            st_vec<4>(da.w + 4 * j, axpy_vec<4>(scale, sum, wv));
+        } else {
+            Vec<4> wv[PT];
+#pragma unroll
+            for (int p = 0; p < PT; ++p) wv[p] = ld_vec<4>(da.w + (int64_t)p * da.w_stride + 4 * j);
+#pragma unroll
+            for (int p = 0; p < PT; ++p) {
+                Vec<4> gh, rs;
+                decode_vec<EF, 4>(v[p][k], c[p], gh, rs);
+                if (STORE) st_vec<4>(da.err + (int64_t)p * da.err_stride + 4 * j, rs);
+                st_vec<4>(da.w + (int64_t)p * da.w_stride + 4 * j, axpy_vec<4>(scale, gh, wv[p]));
+            }
+        }
+    }
+    if (has_tail) {
+        float sum = 0.f;
+#pragma unroll
+        for (int p = 0; p < PT; ++p) {
+            float gh, rs;
+            decode1<EF>(v_tail[p], c[p], gh, rs);
+            if (STORE) st_stream1(da.err + (int64_t)p * da.err_stride + i_tail, rs);
+            if (SHARED) {
+                sum += gh;
+            } else {
+                float *wp = da.w + (int64_t)p * da.w_stride + i_tail;
+                *wp = fmaf(scale, gh, *wp);
+            }
+        }
+        if (SHARED) da.w[i_tail] = fmaf(scale, sum, da.w[i_tail]);
     }
 }
 

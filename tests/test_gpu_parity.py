@@ -64,11 +64,13 @@ SIZES = [1, 2, 3, 4, 5, 31, 32, 33, 127, 1023, 1024, 1025, 4099, 65536 + 7, (1 <
 @pytest.mark.parametrize("n", SIZES)
 def test_single_step_matches_oracle(mode, replicated, n):
     P = [1, 2, 3, 4, 8, 16][(n + int(replicated)) % 6]
-    # worker stride a multiple of 4 elements (vector kernels) except when n % 3 == 0 (scalar kernels)
-    pad = ((-n) % 4) if n % 3 else 1
+    # worker stride chosen so that all three kernel families are hit across the size list:
+    # stride % 8 == 0 -> 256-bit kernels, stride % 8 == 4 -> 128-bit kernels, stride % 4 == 1 -> scalar
+    want = [0, 4, 1][n % 3]
+    pad = (want - n) % 8
     views, raw, stride = _state(1000 + n, P, n, pad=pad, replicated=replicated)
     g, e, w = _host(views)
-    ctx = B.a2sgd_create(n, P, 0, mode)
+    ctx = B.a2sgd_create(n, P, 0, mode | B.FORCE_TWO_PASS)
     # stage 1: encode (means, counts, mask) -- bit-exact integers, 1e-6 means
     lm_buf = torch.full((P + 2, 2), NAN, device="cuda")
     lm = lm_buf[1:P + 1]
@@ -98,7 +100,24 @@ def test_single_step_matches_oracle(mode, replicated, n):
     w_ref, e_ref = w.copy(), e.copy()
     lm_o, gm_o, cnt_o = oracle.step(w_ref, g, e_ref, 0.1, mode=mode)
     assert_state(w_arg.cpu().numpy(), w_ref, e_arg.cpu().numpy(), e_ref, gm_o, f"staged n={n} P={P}")
-    # fused step on the originals: same bits as the staged calls
+    # default context (takes the single-launch path when n*P fits on chip) on second copies
+    ctx2 = B.a2sgd_create(n, P, 0, mode)
+    w2_raw, e2_raw = raw["w"].clone(), raw["e"].clone()
+    w2_view = w2_raw[(views["w"].data_ptr() - raw["w"].data_ptr()) // 4:]
+    e2_view = e2_raw[(views["e"].data_ptr() - raw["e"].data_ptr()) // 4:]
+    w2 = w2_view[:P * stride].view(P, stride)[:, :n] if replicated else w2_view[:n]
+    e2 = e2_view[:P * stride].view(P, stride)[:, :n]
+    B.a2sgd_step(ctx2, w2, views["g"], e2, 0.1)
+    lm_c, gm_c, cnt_c, status = B.a2sgd_read_stats(ctx2)
+    assert status == B.OK and np.array_equal(cnt_c, cnt_ref)
+    assert_means(lm_c, lm_ref, "default step local means")
+    assert_means(gm_c, gm_ref, "default step global means")
+    assert_state(w2.cpu().numpy(), w_ref, e2.cpu().numpy(), e_ref, gm_o, f"default step n={n} P={P}")
+    raw2 = {"g": raw["g"], "e": e2_raw, "w": w2_raw}
+    views2 = {"g": views["g"], "e": e2, "w": w2}
+    _guards_intact(raw2, views2, n, stride, {"g": P, "e": P, "w": P if replicated else 1})
+    ctx2.destroy()
+    # fused two-pass step on the originals: same bits as the staged calls
     B.a2sgd_step(ctx, views["w"], views["g"], views["e"], 0.1)
     lm_s, gm_s, cnt_s, status = B.a2sgd_read_stats(ctx)
     assert status == B.OK
@@ -338,3 +357,78 @@ def test_host_gradient_entry_point():
     assert_means(means[2 * P:].numpy(), gm_ref)
     assert_state(w.cpu().numpy(), w_ref, e.cpu().numpy(), e_ref, gm_ref, "host entry")
     ctx.destroy()
+
+
+@pytest.mark.parametrize("mode", [EF, ALG1])
+@pytest.mark.parametrize("P,n", [(1, 1 << 20), (1, (1 << 20) + 3), (2, 500_001), (4, 250_000), (8, 123_457), (4, 5)])
+@pytest.mark.parametrize("replicated", [False, True])
+def test_single_launch_path(mode, P, n, replicated):
+    """The cooperative single-launch kernel (v kept in registers between the two phases) against
+    the oracle, and forced explicitly so that a silent fall-back to two launches cannot pass."""
+    g = B.padded_rows(P, n, "cuda")
+    e = B.padded_rows(P, n, "cuda")
+    gen = torch.Generator("cuda").manual_seed(n + P)
+    g.normal_(0.0, 1e-3, generator=gen)
+    e.normal_(0.0, 3e-4, generator=gen)
+    w = B.padded_rows(P, n, "cuda") if replicated else torch.empty(n, device="cuda")
+    w.normal_(0.0, 0.02, generator=gen)
+    gh, eh, wh = g.cpu().numpy().copy(), e.cpu().numpy().copy(), w.cpu().numpy().copy()
+    ctx = B.a2sgd_create(n, P, 0, mode | B.FORCE_COOPERATIVE)
+    assert B.a2sgd_launch_info(ctx, shared_w=not replicated)["single_launch"]
+    outs = []
+    for rep in range(2):                     # twice from the same state: bitwise reproducible
+        w_i, e_i = w.clone(), e.clone()
+        if replicated:
+            w_i = B.padded_rows(P, n, "cuda"); w_i.copy_(w)
+        e_pad = B.padded_rows(P, n, "cuda"); e_pad.copy_(e); e_i = e_pad
+        B.a2sgd_step(ctx, w_i, g, e_i, 0.1)
+        lm, gm, cnt, status = B.a2sgd_read_stats(ctx)
+        assert status == B.OK
+        outs.append((lm.tobytes(), gm.tobytes(), cnt.tobytes(), w_i.cpu().numpy().tobytes(), e_i.cpu().numpy().tobytes()))
+    assert outs[0] == outs[1]
+    lm_ref, gm_ref, cnt_ref = oracle.step(wh, gh, eh, 0.1, mode=mode)
+    assert np.array_equal(cnt, cnt_ref)
+    assert_means(lm, lm_ref)
+    assert_means(gm, gm_ref)
+    assert_state(w_i.cpu().numpy(), wh, e_i.cpu().numpy(), eh, gm_ref, f"coop P={P} n={n}")
+    ctx.destroy()
+
+
+def test_single_launch_path_refuses_what_does_not_fit():
+    n, P = 1 << 24, 4
+    g = torch.zeros((P, n), device="cuda")
+    e = torch.zeros((P, n), device="cuda")
+    w = torch.zeros(n, device="cuda")
+    ctx = B.a2sgd_create(n, P, 0, EF | B.FORCE_COOPERATIVE)
+    with pytest.raises(B.A2SGDError) as ei:
+        B.a2sgd_step(ctx, w, g, e, 0.1)
+    assert ei.value.status == B.ERR_TOO_LARGE
+    ctx.destroy()
+    ctx = B.a2sgd_create(1000, 3, 0, EF | B.FORCE_COOPERATIVE)     # P = 3 has no single-launch kernel
+    with pytest.raises(B.A2SGDError):
+        B.a2sgd_step(ctx, w[:1000], g[:3, :1000], e[:3, :1000], 0.1)
+    ctx.destroy()
+
+
+def test_bounded_barrier_wait_times_out_cleanly():
+    """A grid barrier that can never open (the test hook asks for one arrival more than the
+    grid has): every CTA gives up after its poll limit, nothing is written, the status word
+    reports the timeout, and the device stays usable."""
+    n, P = 200_000, 2
+    g = B.padded_rows(P, n, "cuda"); g.normal_(0.0, 1e-3)
+    e = B.padded_rows(P, n, "cuda"); e.normal_(0.0, 1e-4)
+    w = torch.randn(n, device="cuda") * 0.02
+    e0, w0 = e.clone(), w.clone()
+    ctx = B.a2sgd_create(n, P, 0, EF | B.FORCE_COOPERATIVE | B.TEST_BARRIER_NEVER_OPENS)
+    B.a2sgd_step(ctx, w, g, e, 0.1)
+    *_, status = B.a2sgd_read_stats(ctx)
+    assert status == B.ERR_TIMEOUT
+    assert torch.equal(e, e0) and torch.equal(w, w0)
+    *_, status = B.a2sgd_read_stats(ctx)
+    assert status == B.OK
+    ctx.destroy()
+    good = B.a2sgd_create(n, P, 0, EF | B.FORCE_COOPERATIVE)
+    B.a2sgd_step(good, w, g, e, 0.1)
+    *_, status = B.a2sgd_read_stats(good)
+    assert status == B.OK and not torch.equal(w, w0)
+    good.destroy()
