@@ -39,7 +39,8 @@ FALLBACK_HBM_GBS = 6650.0
 
 # DRAM bytes (read + write) per model element of the decode/update kernel, from the ncu
 # captures summarised under profiles/ (None until a capture exists for that P).
-NCU_DECODE_TRAFFIC_PER_ELEMENT = {}
+NCU_DECODE_TRAFFIC_PER_ELEMENT = {4: 52.94}  # 36.0 read + 16.94 written inside the launch; 3.06 B/element of
+#                                               dirty lines leave L2 during the next launch
 
 
 def algorithmic_bytes_per_model_element(P: int, shared_w: bool = True) -> dict:
@@ -186,6 +187,21 @@ def run_reference(args):
 
 
 # ----------------------------------------------------------------------------- device arm
+def max_over_ranks(ms: float, dist, device) -> float:
+    """Every rank contributes its own device-timed milliseconds; all get the maximum."""
+    if dist is None:
+        return ms
+    import torch
+    t = torch.tensor([ms], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(n_model: int, n_replicas: int, ms_per_step: float) -> float:
+    """Model parameters per second summed over the independent replicas."""
+    return n_replicas * n_model / (ms_per_step * 1e-3)
+
+
 def time_workload(wl, steps, warmup, dev, *, with_roofline=True, with_e2e=True, dist=None):
     """Runs the timed regions for one workload on this rank's GPU.  Returns a dict of results."""
     import torch
@@ -244,11 +260,7 @@ def time_workload(wl, steps, warmup, dev, *, with_roofline=True, with_e2e=True, 
     ev1.record()
     barrier()
     wall1 = time.time()
-    ms = ev0.elapsed_time(ev1)
-    if dist is not None:
-        t = torch.tensor([ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    ms = max_over_ranks(ev0.elapsed_time(ev1), dist, dev)
     res = {"ms_total": ms, "ms_per_step": ms / steps, "launches": launches_per_step * steps,
            "launch_info": info, "wall": (wall0, wall1),
            "launch_mode": f"CUDA graph of {chunk} steps" if graph is not None else "eager"}
@@ -293,11 +305,7 @@ def time_workload(wl, steps, warmup, dev, *, with_roofline=True, with_e2e=True, 
             B.a2sgd_step_host(ctx, w, g_host, g, e, wl.lr, means)
         ev1.record()
         barrier()
-        ms2 = ev0.elapsed_time(ev1)
-        if dist is not None:
-            t = torch.tensor([ms2], device=dev, dtype=torch.float64)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms2 = float(t.item())
+        ms2 = max_over_ranks(ev0.elapsed_time(ev1), dist, dev)
         res["e2e_ms_per_step"] = ms2 / e2e_steps
         res["e2e_steps"] = e2e_steps
         res["h2d_bytes"] = P * n * 4
@@ -431,7 +439,7 @@ def main():
 
     b = algorithmic_bytes_per_model_element(wl.P)
     t = res["ms_per_step"] * 1e-3
-    value = n_gpus * wl.n / t
+    value = whole_job_value(wl.n, n_gpus, res["ms_per_step"])
     dec_t = res["decode_ms"] * 1e-3
     achieved = b["decode"] * wl.n / dec_t / 1e9
     traffic_per_el = NCU_DECODE_TRAFFIC_PER_ELEMENT.get(wl.P)

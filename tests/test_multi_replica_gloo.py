@@ -1,0 +1,66 @@
+"""Host-side logic of the multi-GPU benchmark mode, on CPU with gloo (world size 2).
+
+The measured path has no exchange between GPUs, so N GPUs run N independent replicas; what
+the ranks share is only the timing protocol: barrier, max over ranks of the device time, and
+rank 0 reporting the whole-job value."""
+import os
+import socket
+import subprocess
+import sys
+import textwrap
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _free_port():
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+WORKER = textwrap.dedent("""
+    import os, sys
+    sys.path.insert(0, {root!r})
+    import torch
+    import torch.distributed as dist
+    import bench
+    dist.init_process_group("gloo", init_method="tcp://127.0.0.1:{port}", rank=int(sys.argv[1]), world_size=2)
+    rank = dist.get_rank()
+    dist.barrier()
+    ms_local = 10.0 + 5.0 * rank                      # rank 1 is the slow one
+    ms = bench.max_over_ranks(ms_local, dist, torch.device("cpu"))
+    assert ms == 15.0, ms
+    value = bench.whole_job_value(1000, dist.get_world_size(), ms)
+    assert abs(value - 2 * 1000 / 15e-3) < 1e-6
+    dist.barrier()
+    dist.destroy_process_group()
+    print("rank", rank, "ok")
+""")
+
+
+def test_max_over_ranks_and_whole_job_value_world_size_2(tmp_path):
+    port = _free_port()
+    script = tmp_path / "worker.py"
+    script.write_text(WORKER.format(root=ROOT, port=port))
+    procs = [subprocess.Popen([sys.executable, str(script), str(r)], stdout=subprocess.PIPE,
+                              stderr=subprocess.STDOUT, text=True) for r in range(2)]
+    outs = [p.communicate(timeout=180)[0] for p in procs]
+    for r, (p, out) in enumerate(zip(procs, outs)):
+        assert p.returncode == 0, out
+        assert f"rank {r} ok" in out
+
+
+def test_reference_arm_prints_only_on_rank_zero():
+    env = dict(os.environ, RANK="1", WORLD_SIZE="2")
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--gpus", "2",
+                          "--steps", "1", "--warmup", "0"], env=env, capture_output=True, text=True, timeout=300)
+    assert out.returncode == 0 and out.stdout.strip() == ""
+
+
+def test_single_rank_passthrough():
+    sys.path.insert(0, ROOT)
+    import bench
+    assert bench.max_over_ranks(3.5, None, None) == 3.5
+    assert bench.algorithmic_bytes_per_model_element(4) == {"encode": 32, "decode": 56, "step": 88}
+    assert bench.algorithmic_bytes_per_model_element(8)["step"] == 168
+    assert bench.algorithmic_bytes_per_model_element(1)["step"] == 28
