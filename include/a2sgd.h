@@ -153,6 +153,32 @@ int a2sgd_read_stats(a2sgd_ctx *ctx, float *local_means_host,
  * path for this (n, P), out[4] = SM count.  HOST pointer. */
 int a2sgd_launch_info(a2sgd_ctx *ctx, int64_t w_stride, uint32_t out[5]);
 
+/* The encode step (two local means per worker, see a2sgd_encode) for callers that must not
+ * allocate device memory.  The paper has no counterpart to this entry point: it exists for
+ * integration reasons only.  Typical callers: code running inside a framework that has given
+ * the whole GPU to its own caching allocator (a raw cudaMalloc there fails or fragments the
+ * pool), loops that cannot afford the device-wide synchronisation a cudaMalloc implies, and
+ * plug-ins bound by a "nothing is allocated after start-up" rule.  It takes no context: the
+ * reduction scratch is a fixed 64 KiB array inside the library image (every GPU that loads the
+ * library holds it until the process exits), and the call itself performs no cudaMalloc,
+ * cudaFree or other allocating call.
+ *   n, P         as in a2sgd_create; P <= A2SGD_NOALLOC_MAX_P, else A2SGD_ERR_TOO_LARGE
+ *                (the fixed scratch has ticket slots for that many workers; n is not limited
+ *                beyond n < 2^40 because the grid, not n, sizes the partial sums)
+ *   mode         A2SGD_MODE_EF or A2SGD_MODE_ALG1
+ *   grad, err    device, as in a2sgd_encode (err required in EF mode)
+ *   local_means  device, out, [P][2];  pos_counts  device, out, [P], may be NULL
+ * Runs on the CURRENT device.  The first call on each device also looks up the device address of
+ * the scratch array; make that first call before any stream capture begins.  All calls on a
+ * device share the one scratch array: the tickets are cleared at the start of every call, but two
+ * calls whose kernels overlap on the GPU (different streams, different threads) race on it and
+ * give wrong means — serialise them.  No packed mask output and no latched device status here;
+ * results are identical to a2sgd_encode up to the summation order of a differently sized grid. */
+#define A2SGD_NOALLOC_MAX_P 64
+int a2sgd_encode_noalloc(uint64_t n, uint32_t P, uint32_t mode, const float *grad, int64_t grad_stride,
+                         const float *err, int64_t err_stride, float *local_means, uint64_t *pos_counts,
+                         void *stream);
+
 /* Static, never NULL. */
 const char *a2sgd_status_string(int status);
 

@@ -67,6 +67,9 @@ def lib() -> ctypes.CDLL:
         l.a2sgd_read_stats.argtypes = [_vp, _vp, _vp, _vp, ctypes.POINTER(ctypes.c_int), _vp]
         l.a2sgd_launch_info.restype = ctypes.c_int
         l.a2sgd_launch_info.argtypes = [_vp, _i64, ctypes.POINTER(ctypes.c_uint32)]
+        l.a2sgd_encode_noalloc.restype = ctypes.c_int
+        l.a2sgd_encode_noalloc.argtypes = [ctypes.c_uint64, ctypes.c_uint32, ctypes.c_uint32, _vp, _i64, _vp, _i64,
+                                           _vp, _vp, _vp]
         l.a2sgd_status_string.restype = ctypes.c_char_p
         l.a2sgd_status_string.argtypes = [ctypes.c_int]
         _lib = l
@@ -161,6 +164,25 @@ def a2sgd_encode(ctx: Context, grad: torch.Tensor, err: Optional[torch.Tensor], 
                               pos_counts.data_ptr() if pos_counts is not None else None,
                               pos_mask.data_ptr() if pos_mask is not None else None, _stream(stream)),
            "a2sgd_encode")
+
+
+NOALLOC_MAX_P = 64
+
+
+def a2sgd_encode_noalloc(grad: torch.Tensor, err: Optional[torch.Tensor], local_means: torch.Tensor,
+                         pos_counts: Optional[torch.Tensor] = None, mode: int = MODE_EF, n: Optional[int] = None,
+                         stream=None) -> None:
+    """Encode without a context and without any allocation inside the library (its scratch is a
+    fixed array in the library image).  For callers that may not call cudaMalloc; runs on the
+    current device; calls that overlap on the GPU race on the shared scratch.  Output tensors are
+    the caller's: local_means float32 CUDA [P, 2], pos_counts int64 CUDA [P]."""
+    gp, gs = _rows(grad, "grad")
+    ep, es = _rows(err, "err")
+    P = grad.shape[0]
+    n = grad.shape[1] if n is None else n
+    _check(lib().a2sgd_encode_noalloc(int(n), int(P), int(mode), gp, gs, ep, es, local_means.data_ptr(),
+                                      pos_counts.data_ptr() if pos_counts is not None else None,
+                                      _stream(stream)), "a2sgd_encode_noalloc")
 
 
 def a2sgd_global_average(ctx: Context, local_means: torch.Tensor, global_means: torch.Tensor, stream=None) -> None:

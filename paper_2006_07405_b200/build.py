@@ -12,7 +12,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "liba2sgd.so")
-SOURCES = [os.path.join(CSRC, "a2sgd.cu")]
+SOURCES = [os.path.join(CSRC, "a2sgd.cu"), os.path.join(CSRC, "a2sgd_noalloc.cu")]
 DEPENDS = SOURCES + [os.path.join(CSRC, "a2sgd_kernels.cuh"), os.path.join(ROOT, "include", "a2sgd.h")]
 
 NVCC_FLAGS = [

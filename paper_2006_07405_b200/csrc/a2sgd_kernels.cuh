@@ -417,7 +417,7 @@ __global__ void __launch_bounds__(kBlock) k_encode_scalar(EncodeArgs a)
 }
 
 // ------------------------------------------------------------------ K2: global average (stand-alone form)
-__global__ void k_global_average(const float *__restrict__ local_means, uint32_t P, float *global_means,
+static __global__ void k_global_average(const float *__restrict__ local_means, uint32_t P, float *global_means,
                                  float *ctx_global_means)
 {
     if (threadIdx.x != 0 || blockIdx.x != 0) return;
