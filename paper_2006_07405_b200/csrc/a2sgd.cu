@@ -13,6 +13,19 @@
 
 using namespace a2sgd;
 
+// Grid shapes (measured on B200, CUDA events, c2/c3/c4 workloads):
+//  * decode: one vector per thread, as many CTAs as that takes.  A persistent grid of
+//    148 x occupancy CTAs with an equal static share each ran the same kernel at 6.2 TB/s; the
+//    SMs do not stream at equal speed (two dies, shared channels), so the slowest share set the
+//    time.  Letting the hardware CTA scheduler hand out small CTAs reaches 6.9-7.0 TB/s.
+//  * encode: per-CTA partial sums must stay few and their order fixed, so the grid stays
+//    proportional to the resident-CTA count; two CTAs per resident slot is the best measured.
+#ifndef A2SGD_WAVES_K1
+#define A2SGD_WAVES_K1 2
+#endif
+#ifndef A2SGD_WAVES_K3
+#define A2SGD_WAVES_K3 (1 << 20) /* effectively: cover every vector with its own thread */
+#endif
 #ifndef A2SGD_MAX_VW
 #define A2SGD_MAX_VW 8 /* widest vector access the dispatcher may pick: 8 = 256-bit, 4 = 128-bit */
 #endif
@@ -81,6 +94,26 @@ inline int vec_width(const void *p, int64_t stride, uint32_t P)
     return 0;
 }
 
+#ifndef A2SGD_PDL
+#define A2SGD_PDL 1
+#endif
+
+// Launch with programmatic stream serialisation (see pdl_wait_prior_grid in the kernels).
+cudaError_t launch_pdl(const void *fn, dim3 grid, void **params, cudaStream_t s)
+{
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = grid;
+    cfg.blockDim = dim3(kBlock);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = A2SGD_PDL;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelExC(&cfg, fn, params);
+}
+
 int occupancy(a2sgd_ctx *c, const void *kernel)
 {
     auto it = c->occ.find(kernel);
@@ -96,20 +129,20 @@ int occupancy(a2sgd_ctx *c, const void *kernel)
 }
 
 // CTAs per worker for a (G, P) grid that fills the device exactly once.
-inline uint32_t per_worker_grid(const a2sgd_ctx *c, int occ, uint64_t items)
+inline uint32_t per_worker_grid(const a2sgd_ctx *c, int occ, uint64_t items, int waves = 1)
 {
-    const uint64_t slots = (uint64_t)c->sm_count * (uint64_t)std::max(occ, 1);
+    const uint64_t slots = (uint64_t)c->sm_count * (uint64_t)std::max(occ, 1) * (uint64_t)waves;
     uint64_t G = std::max<uint64_t>(1, slots / c->P);
     const uint64_t need = std::max<uint64_t>(1, (items + kBlock - 1) / kBlock);
     G = std::min(G, need);
-    return (uint32_t)std::min<uint64_t>(G, c->g_alloc);
+    return (uint32_t)std::min<uint64_t>(G, 0x7fffffffu);
 }
 
-inline uint32_t flat_grid(const a2sgd_ctx *c, int occ, uint64_t items)
+inline uint32_t flat_grid(const a2sgd_ctx *c, int occ, uint64_t items, int waves = 1)
 {
-    const uint64_t slots = (uint64_t)c->sm_count * (uint64_t)std::max(occ, 1);
+    const uint64_t slots = (uint64_t)c->sm_count * (uint64_t)std::max(occ, 1) * (uint64_t)waves;
     const uint64_t need = std::max<uint64_t>(1, (items + kBlock - 1) / kBlock);
-    return (uint32_t)std::min(slots, need);
+    return (uint32_t)std::min<uint64_t>(std::min(slots, need), 0x7fffffffu);
 }
 
 // ---------------------------------------------------------------- kernel selection
@@ -244,9 +277,9 @@ int launch_encode(a2sgd_ctx *c, const float *grad, int64_t gs, const float *err,
     EncodeArgs a = make_encode_args(c, grad, gs, err, es, local_means, pos_counts, pos_mask, global_means);
     const void *fn = select_encode(!c->alg1, pos_mask != nullptr, vw);
     const uint64_t items = vw ? (c->n + vw - 1) / vw : c->n;
-    const dim3 grid(per_worker_grid(c, occupancy(c, fn), items), c->P);
+    const dim3 grid(std::min(per_worker_grid(c, occupancy(c, fn), items, A2SGD_WAVES_K1), c->g_alloc), c->P);
     void *params[] = {&a};
-    A2_CUDA(cudaLaunchKernel(fn, grid, dim3(kBlock), params, 0, s));
+    A2_CUDA(launch_pdl(fn, grid, params, s));
     return A2SGD_OK;
 }
 
@@ -264,16 +297,16 @@ int launch_decode(a2sgd_ctx *c, float *w, int64_t ws, const float *grad, int64_t
     dim3 grid;
     if (vw && shared) {
         fn = select_decode_shared(ef, store, c->P, vw);
-        grid = dim3(flat_grid(c, occupancy(c, fn), (c->n + vw - 1) / vw));
+        grid = dim3(flat_grid(c, occupancy(c, fn), (c->n + vw - 1) / vw, A2SGD_WAVES_K3));
     } else if (vw) {
         fn = select_decode_repl(ef, store, vw);
-        grid = dim3(per_worker_grid(c, occupancy(c, fn), (c->n + vw - 1) / vw), c->P);
+        grid = dim3(per_worker_grid(c, occupancy(c, fn), (c->n + vw - 1) / vw, A2SGD_WAVES_K3), c->P);
     } else {
         fn = select_decode_scalar(ef, store);
-        grid = shared ? dim3(flat_grid(c, occupancy(c, fn), c->n), 1)
-                      : dim3(per_worker_grid(c, occupancy(c, fn), c->n), c->P);
+        grid = shared ? dim3(flat_grid(c, occupancy(c, fn), c->n, A2SGD_WAVES_K3), 1)
+                      : dim3(per_worker_grid(c, occupancy(c, fn), c->n, A2SGD_WAVES_K3), c->P);
     }
-    A2_CUDA(cudaLaunchKernel(fn, grid, dim3(kBlock), params, 0, s));
+    A2_CUDA(launch_pdl(fn, grid, params, s));
     return A2SGD_OK;
 }
 
@@ -358,7 +391,7 @@ extern "C" int a2sgd_create(a2sgd_ctx **out, uint64_t n, uint32_t P, int device,
         c->coop_supported = coop != 0;
     }
     // partials: room for a (G, P) grid that fills the device at the highest possible occupancy
-    const uint32_t max_slots = (uint32_t)c->sm_count * (2048 / kBlock);
+    const uint32_t max_slots = (uint32_t)c->sm_count * (2048 / kBlock) * A2SGD_WAVES_K1;
     c->g_alloc = std::max<uint32_t>(1, max_slots / P);
     bool ok = true;
     ok = ok && cudaMalloc(&c->partials, sizeof(Partial) * (size_t)c->g_alloc * P) == cudaSuccess;
@@ -534,9 +567,10 @@ extern "C" int a2sgd_launch_info(a2sgd_ctx *c, int64_t w_stride, uint32_t out[5]
     const bool shared = w_stride == 0 || c->P == 1;
     const int vw = A2SGD_MAX_VW >= 8 ? 8 : 4;
     const uint64_t items = (c->n + vw - 1) / vw;
-    out[0] = per_worker_grid(c, occupancy(c, select_encode(ef, false, vw)), items) * c->P;
-    out[1] = shared ? flat_grid(c, occupancy(c, select_decode_shared(ef, true, c->P, vw)), items)
-                    : per_worker_grid(c, occupancy(c, select_decode_repl(ef, true, vw)), items) * c->P;
+    out[0] = std::min(per_worker_grid(c, occupancy(c, select_encode(ef, false, vw)), items, A2SGD_WAVES_K1),
+                      c->g_alloc) * c->P;
+    out[1] = shared ? flat_grid(c, occupancy(c, select_decode_shared(ef, true, c->P, vw)), items, A2SGD_WAVES_K3)
+                    : per_worker_grid(c, occupancy(c, select_decode_repl(ef, true, vw)), items, A2SGD_WAVES_K3) * c->P;
     out[2] = kBlock;
     out[3] = 0;
     if (!(c->flags & A2SGD_FORCE_TWO_PASS)) {

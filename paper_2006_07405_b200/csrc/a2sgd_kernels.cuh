@@ -9,9 +9,13 @@
 //                     (Algorithm 1 lines 4, 6, 7), one streaming pass.
 //
 // Everything here is bound by HBM bandwidth, so the kernels are built around
-// 128-bit coalesced accesses with many independent loads in flight per
-// thread, persistent grids sized to the SM count, streaming cache policy, and
-// no tensor cores (nothing on this path is a contraction).
+// 128/256-bit coalesced accesses with many independent loads in flight per
+// thread, streaming cache policy, and no tensor cores (nothing on this path
+// is a contraction).  Grids: the reduction kernels run a few CTAs per
+// resident slot with grid-stride loops (few, fixed-order partial sums); the
+// element-wise decode kernels are launched with one vector per thread, which
+// lets the hardware CTA scheduler even out SMs that stream at different
+// speeds (the host picks the grid; the loops here accept any grid).
 //
 // Summation.  Within one unrolled batch a thread adds non-negative fp32
 // values pairwise (depth <= 4, relative error <= 4 * 2^-24 of the batch sum);
@@ -42,6 +46,21 @@ struct __align__(8) Partial {
     double s_neg;
     unsigned long long n_pos;
 };
+
+// ------------------------------------------------------------------ programmatic dependent launch
+// The two kernels of a step (and the steps of a loop) are launched with programmatic stream
+// serialisation: a kernel's CTAs may become resident while the previous kernel drains, which
+// hides the launch latency at each kernel boundary.  Every kernel therefore waits for the
+// previous grid (completion and memory flush) before its first global access, and then lets
+// its own successor start being scheduled.
+__device__ __forceinline__ void pdl_wait_prior_grid()
+{
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+__device__ __forceinline__ void pdl_release_next_grid()
+{
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
 
 // ------------------------------------------------------------------ memory access helpers
 // Streaming vector accesses, VW = 4 (128-bit) or 8 (256-bit, new on sm_100).
@@ -284,6 +303,9 @@ __device__ __forceinline__ void finish_worker(const EncodeArgs &a, uint32_t p, d
 template <bool EF, bool MASK, int VW>
 __global__ void __launch_bounds__(kBlock) k_encode_vec(EncodeArgs a)
 {
+    pdl_wait_prior_grid();
+    pdl_release_next_grid();
+
     constexpr int LPW = 32 / VW;  // lanes per mask word
     constexpr int U = 16 / VW;    // vectors per trip: 16 elements per thread per batch
     __shared__ double sh_d[2][kWarps];
@@ -384,6 +406,9 @@ __global__ void __launch_bounds__(kBlock) k_encode_vec(EncodeArgs a)
 template <bool EF, bool MASK>
 __global__ void __launch_bounds__(kBlock) k_encode_scalar(EncodeArgs a)
 {
+    pdl_wait_prior_grid();
+    pdl_release_next_grid();
+
     __shared__ double sh_d[2][kWarps];
     __shared__ unsigned long long sh_n[kWarps];
     __shared__ int sh_flag;
@@ -420,6 +445,9 @@ __global__ void __launch_bounds__(kBlock) k_encode_scalar(EncodeArgs a)
 static __global__ void k_global_average(const float *__restrict__ local_means, uint32_t P, float *global_means,
                                  float *ctx_global_means)
 {
+    pdl_wait_prior_grid();
+    pdl_release_next_grid();
+
     if (threadIdx.x != 0 || blockIdx.x != 0) return;
     double gp = 0.0, gn = 0.0;
     for (uint32_t q = 0; q < P; ++q) { // worker order
@@ -524,6 +552,9 @@ __device__ __forceinline__ Vec<VW> zero_vec()
 template <bool EF, bool STORE, int PT, int VW>
 __global__ void __launch_bounds__(kBlock) k_decode_shared_vec(DecodeArgs a)
 {
+    pdl_wait_prior_grid();
+    pdl_release_next_grid();
+
     __shared__ WorkerConst sh_c[PT > 0 ? 1 : kMaxP];
     const uint32_t P = PT > 0 ? PT : a.P;
     const float m_pos = __ldg(a.global_means), m_neg = __ldg(a.global_means + 1);
@@ -596,6 +627,9 @@ __global__ void __launch_bounds__(kBlock) k_decode_shared_vec(DecodeArgs a)
 template <bool EF, bool STORE, int VW>
 __global__ void __launch_bounds__(kBlock) k_decode_repl_vec(DecodeArgs a)
 {
+    pdl_wait_prior_grid();
+    pdl_release_next_grid();
+
     const uint32_t p = blockIdx.y;
     const float m_pos = __ldg(a.global_means), m_neg = __ldg(a.global_means + 1);
     const WorkerConst c = worker_const<EF>(a, p, m_pos, m_neg);
@@ -653,6 +687,9 @@ __global__ void __launch_bounds__(kBlock) k_decode_repl_vec(DecodeArgs a)
 template <bool EF, bool STORE>
 __global__ void __launch_bounds__(kBlock) k_decode_scalar(DecodeArgs a)
 {
+    pdl_wait_prior_grid();
+    pdl_release_next_grid();
+
     const float m_pos = __ldg(a.global_means), m_neg = __ldg(a.global_means + 1);
     const uint64_t stride = (uint64_t)gridDim.x * kBlock;
     const bool shared = a.w_stride == 0;
