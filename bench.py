@@ -39,7 +39,7 @@ FALLBACK_HBM_GBS = 6650.0
 
 # DRAM bytes (read + write) per model element of the decode/update kernel, from the ncu
 # captures summarised under profiles/ (None until a capture exists for that P).
-NCU_DECODE_TRAFFIC_PER_ELEMENT = {4: 52.94}  # 36.0 read + 16.94 written inside the launch; 3.06 B/element of
+NCU_DECODE_TRAFFIC_PER_ELEMENT = {4: 52.92}  # 36.0 read + 16.92 written inside the launch; 3.08 B/element of
 #                                               dirty lines leave L2 during the next launch
 
 
