@@ -61,6 +61,9 @@ def _load():
             ctypes.c_int, ctypes.c_uint64, ctypes.c_uint32, f32p, ctypes.c_int64,
             f32p, ctypes.c_int64, f32p, ctypes.c_int64, ctypes.c_float,
             f32p, f32p, u64p]
+        lib.a2sgd_oracle_dense_sync.restype = ctypes.c_int
+        lib.a2sgd_oracle_dense_sync.argtypes = [
+            ctypes.c_uint64, ctypes.c_uint32, f32p, ctypes.c_int64, f32p, ctypes.c_int64, ctypes.c_float]
         _lib = lib
     return _lib
 
@@ -152,3 +155,13 @@ def step(w, grad, err, lr, *, mode=MODE_EF, n=None):
         gmeans.ctypes.data_as(ctypes.POINTER(ctypes.c_float)),
         counts.ctypes.data_as(ctypes.POINTER(ctypes.c_uint64))), "step")
     return means, gmeans, counts
+
+
+def dense_sync(w, grad, lr, *, n=None):
+    """Algorithm 1 lines 9-10: w <- w - lr * mean over workers of grad, in place."""
+    lib = _load()
+    P = grad.shape[0]
+    n = grad.shape[1] if n is None else n
+    gp, gs = _rows(grad, "grad")
+    wp, ws = _weights(w, P)
+    _check(lib.a2sgd_oracle_dense_sync(n, P, wp, ws, gp, gs, lr), "dense_sync")

@@ -170,6 +170,32 @@ int a2sgd_oracle_decode_update(int mode, uint64_t n, uint32_t P,
     return 0;
 }
 
+/*
+ * Algorithm 1 lines 9-10: after the last compressed iteration one dense
+ * synchronisation — the workers' gradients are averaged element-wise
+ * (Allreduce-average of the full vectors) and every worker applies
+ * w <- w - lr * mean_p g^p.  This is Eq. 1 (dense distributed SGD) for one
+ * step.  w_stride == 0: one shared w; otherwise every replica receives the
+ * same averaged update.
+ */
+int a2sgd_oracle_dense_sync(uint64_t n, uint32_t P, float *w, int64_t w_stride,
+                            const float *grad, int64_t grad_stride, float lr)
+{
+    if (n == 0 || P == 0 || !w || !grad) return -1;
+    const uint32_t replicas = (w_stride == 0) ? 1 : P;
+    for (uint64_t i = 0; i < n; ++i) {
+        double sum = 0.0;
+        for (uint32_t p = 0; p < P; ++p)
+            sum += (double)grad[(int64_t)p * grad_stride + (int64_t)i];
+        const double mean = sum / (double)P;
+        for (uint32_t r = 0; r < replicas; ++r) {
+            float *wr = w + (int64_t)r * w_stride;
+            wr[i] = (float)((double)wr[i] - (double)lr * mean);
+        }
+    }
+    return 0;
+}
+
 /* One whole iteration of the loop body of Algorithm 1 for all P workers. */
 int a2sgd_oracle_step(int mode, uint64_t n, uint32_t P,
                       float *w, int64_t w_stride,

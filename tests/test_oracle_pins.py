@@ -378,3 +378,49 @@ def test_rejects_bad_arguments():
         oracle.encode(g, None, mode=EF)            # EF needs the error buffer
     with pytest.raises(ValueError):
         oracle.encode(g.astype(np.float64), None, mode=ALG1)
+
+
+# ---------------------------------------------------------------- Algorithm 1 lines 9-10 (dense step)
+def test_dense_sync_matches_numpy_mean_axpy_and_special_cases():
+    rng = np.random.default_rng(31)
+    P, n, lr = 5, 20011, 0.3
+    g = (rng.standard_normal((P, n)) * 1e-2).astype(np.float32)
+    w0 = (rng.standard_normal(n) * 0.02).astype(np.float32)
+    ref = w0.astype(np.float64) - np.float64(np.float32(lr)) * g.astype(np.float64).mean(axis=0)
+    w = w0.copy()
+    oracle.dense_sync(w, g, lr)
+    assert np.max(np.abs(w - ref)) <= 1.01 * np.spacing(np.abs(w0).max())
+    # every replica receives the same averaged update (this is what re-synchronises the workers)
+    w_rep = np.tile(w0, (P, 1)) + np.arange(P, dtype=np.float32)[:, None]
+    oracle.dense_sync(w_rep, g, lr)
+    for p in range(P):
+        assert np.max(np.abs(w_rep[p] - (ref + p))) <= 1.01 * np.spacing(np.float32(p + 1))
+    # P = 1 is plain SGD; identical workers give the single-worker result
+    w1 = w0.copy()
+    oracle.dense_sync(w1, g[:1], lr)
+    ref1 = w0.astype(np.float64) - np.float64(np.float32(lr)) * g[0].astype(np.float64)
+    assert np.max(np.abs(w1 - ref1)) <= 1.01 * np.spacing(np.abs(w0).max())
+    w2 = w0.copy()
+    oracle.dense_sync(w2, np.tile(g[:1], (4, 1)), lr)
+    assert np.array_equal(w2, w1)
+
+
+@pytest.mark.parametrize("seed", range(10))
+def test_dense_sync_bruteforce_rational(seed):
+    rng = np.random.default_rng(seed)
+    n, P = int(rng.integers(1, 9)), int(rng.integers(1, 6))
+    g = rng.standard_normal((P, n)).astype(np.float32)
+    w0 = rng.standard_normal(n).astype(np.float32)
+    w = w0.copy()
+    oracle.dense_sync(w, g, 0.125)
+    for i in range(n):
+        mean = sum((Fraction(float(g[p, i])) for p in range(P)), Fraction(0)) / P
+        assert _ulp_close(w[i], _round32(Fraction(float(w0[i])) - Fraction(1, 8) * mean))
+
+
+def test_dense_sync_after_identical_local_steps_equals_eq1():
+    """Eq. 1: one dense step from a common w is w - lr * (1/P) sum_p g^p; with hand numbers."""
+    g = _f32([[1, -2, 4], [3, 2, -8]])
+    w = np.array([10, 10, 10], np.float32)
+    oracle.dense_sync(w, g, 0.5)
+    assert w.tolist() == [9.0, 10.0, 11.0]
