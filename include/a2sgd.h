@@ -125,6 +125,15 @@ int a2sgd_step(a2sgd_ctx *ctx, float *w, int64_t w_stride,
                const float *grad, int64_t grad_stride,
                float *err, int64_t err_stride, float lr, void *stream);
 
+/* Algorithm 1 lines 9-10: the dense synchronisation that follows the last compressed iteration
+ * (Eq. 1 for one step).  The workers' gradients are averaged element-wise, summed in worker
+ * order, and applied: w <- w - lr * (1/P) * sum_p grad^p.  With w_stride == 0 the one shared w is
+ * updated; with w_stride >= n every replica receives the same averaged update (which is what
+ * brings drifted replicas back in step).  No error buffer is involved.  One streaming pass:
+ * (4P + 8) bytes per model element for a shared w. */
+int a2sgd_dense_sync(a2sgd_ctx *ctx, float *w, int64_t w_stride,
+                     const float *grad, int64_t grad_stride, float lr, void *stream);
+
 /* a2sgd_step for a caller whose fresh gradients sit in HOST memory (pinned
  * memory makes the copies asynchronous): copies grad_host -> grad_staging
  * worker by worker, runs the step, copies the 2P local and 2 global means

@@ -70,6 +70,8 @@ def lib() -> ctypes.CDLL:
         l.a2sgd_encode_noalloc.restype = ctypes.c_int
         l.a2sgd_encode_noalloc.argtypes = [ctypes.c_uint64, ctypes.c_uint32, ctypes.c_uint32, _vp, _i64, _vp, _i64,
                                            _vp, _vp, _vp]
+        l.a2sgd_dense_sync.restype = ctypes.c_int
+        l.a2sgd_dense_sync.argtypes = [_vp, _vp, _i64, _vp, _i64, ctypes.c_float, _vp]
         l.a2sgd_status_string.restype = ctypes.c_char_p
         l.a2sgd_status_string.argtypes = [ctypes.c_int]
         _lib = l
@@ -208,6 +210,13 @@ def a2sgd_step(ctx: Context, w: torch.Tensor, grad: torch.Tensor, err: Optional[
     gp, gs = _rows(grad, "grad")
     ep, es = _rows(err, "err")
     _check(lib().a2sgd_step(ctx.handle, wp, ws, gp, gs, ep, es, float(lr), _stream(stream)), "a2sgd_step")
+
+
+def a2sgd_dense_sync(ctx: Context, w: torch.Tensor, grad: torch.Tensor, lr: float, stream=None) -> None:
+    """Algorithm 1 lines 9-10: w <- w - lr * mean over workers of grad."""
+    wp, ws = _weights(w)
+    gp, gs = _rows(grad, "grad")
+    _check(lib().a2sgd_dense_sync(ctx.handle, wp, ws, gp, gs, float(lr), _stream(stream)), "a2sgd_dense_sync")
 
 
 def a2sgd_step_host(ctx: Context, w: torch.Tensor, grad_host: torch.Tensor, grad_staging: torch.Tensor,

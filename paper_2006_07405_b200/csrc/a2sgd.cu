@@ -194,6 +194,25 @@ const void *select_decode_scalar(bool ef, bool store)
     return store ? (const void *)k_decode_scalar<false, true> : (const void *)k_decode_scalar<false, false>;
 }
 
+template <int VW, bool REPL>
+const void *select_dense_p(uint32_t P)
+{
+    switch (P) {
+    case 1: return (const void *)k_dense_sync_vec<1, VW, REPL>;
+    case 2: return (const void *)k_dense_sync_vec<2, VW, REPL>;
+    case 4: return (const void *)k_dense_sync_vec<4, VW, REPL>;
+    case 8: return (const void *)k_dense_sync_vec<8, VW, REPL>;
+    default: return (const void *)k_dense_sync_vec<0, VW, REPL>;
+    }
+}
+
+const void *select_dense(uint32_t P, int vw, bool repl)
+{
+    if (vw == 8) return repl ? select_dense_p<8, true>(P) : select_dense_p<8, false>(P);
+    if (vw == 4) return repl ? select_dense_p<4, true>(P) : select_dense_p<4, false>(P);
+    return (const void *)k_dense_sync_scalar;
+}
+
 template <bool EF, bool STORE, bool SHARED>
 const void *select_coop_p(uint32_t P)
 {
@@ -503,6 +522,33 @@ extern "C" int a2sgd_step(a2sgd_ctx *c, float *w, int64_t w_stride, const float 
                                  c->global_means, s);
     if (r1) return r1;
     return launch_decode(c, w, ws, grad, grad_stride, err, err_stride, c->local_means, c->global_means, lr, s);
+}
+
+extern "C" int a2sgd_dense_sync(a2sgd_ctx *c, float *w, int64_t w_stride, const float *grad, int64_t grad_stride,
+                               float lr, void *stream)
+{
+    if (!c || !w || !grad) return A2SGD_ERR_ARG;
+    if (!stride_ok(grad_stride, c->n, c->P)) return A2SGD_ERR_ARG;
+    if (w_stride != 0 && !stride_ok(w_stride, c->n, c->P)) return A2SGD_ERR_ARG;
+    if (!aligned(w, 4) || !aligned(grad, 4)) return A2SGD_ERR_ALIGN;
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return A2SGD_ERR_CUDA;
+    const int64_t ws = (c->P == 1) ? 0 : w_stride;
+    const int vw = std::min(vec_width(grad, grad_stride, c->P), vec_width(w, ws == 0 ? 8 : ws, c->P));
+    DenseArgs a{};
+    a.w = w;
+    a.w_stride = ws;
+    a.grad = grad;
+    a.grad_stride = grad_stride;
+    a.n = c->n;
+    a.P = c->P;
+    a.lr = lr;
+    const void *fn = select_dense(c->P, vw, ws != 0);
+    const uint64_t items = vw ? (c->n + vw - 1) / vw : c->n;
+    const dim3 grid(flat_grid(c, occupancy(c, fn), items, A2SGD_WAVES_K3));
+    void *params[] = {&a};
+    A2_CUDA(launch_pdl(fn, grid, params, static_cast<cudaStream_t>(stream)));
+    return A2SGD_OK;
 }
 
 extern "C" int a2sgd_step_host(a2sgd_ctx *c, float *w, int64_t w_stride, const float *grad_host,

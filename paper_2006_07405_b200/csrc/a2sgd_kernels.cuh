@@ -711,6 +711,83 @@ __global__ void __launch_bounds__(kBlock) k_decode_scalar(DecodeArgs a)
     }
 }
 
+// ------------------------------------------------------------------ K5: dense synchronisation step
+// Algorithm 1 lines 9-10 (Eq. 1 for one step): w <- w - lr * (1/P) sum_p g^p.
+// One streaming pass: P gradient vectors in, summed in worker order, w updated.
+// Shared w: (4P + 8) B per model element; replicas (REPL): every replica gets
+// the same averaged update, (4P + 8P) B.  One vector per thread.
+struct DenseArgs {
+    float *w;
+    int64_t w_stride; // 0 = shared
+    const float *grad;
+    int64_t grad_stride;
+    uint64_t n;
+    uint32_t P;
+    float lr;
+};
+
+template <int PT, int VW, bool REPL>
+__global__ void __launch_bounds__(kBlock) k_dense_sync_vec(DenseArgs a)
+{
+    pdl_wait_prior_grid();
+    pdl_release_next_grid();
+    const uint32_t P = PT > 0 ? PT : a.P;
+    const float scale = -a.lr / (float)P;
+    const uint64_t nv = a.n / VW;
+    const uint64_t stride = (uint64_t)gridDim.x * kBlock;
+    for (uint64_t j = (uint64_t)blockIdx.x * kBlock + threadIdx.x; j < nv; j += stride) {
+        Vec<VW> sum = zero_vec<VW>();
+        if (PT > 0) {
+            constexpr int PP = PT > 0 ? PT : 1;
+            Vec<VW> gv[PP];
+#pragma unroll
+            for (int p = 0; p < PP; ++p) gv[p] = ld_vec<VW>(a.grad + (int64_t)p * a.grad_stride + VW * j);
+#pragma unroll
+            for (int p = 0; p < PP; ++p) sum = add_vec<VW>(sum, gv[p]);
+        } else {
+            for (uint32_t p = 0; p < P; ++p) sum = add_vec<VW>(sum, ld_vec<VW>(a.grad + (int64_t)p * a.grad_stride + VW * j));
+        }
+        if (REPL) {
+            for (uint32_t p = 0; p < P; ++p) {
+                float *wp = a.w + (int64_t)p * a.w_stride + VW * j;
+                st_vec<VW>(wp, axpy_vec<VW>(scale, sum, ld_vec<VW>(wp)));
+            }
+        } else {
+            st_vec<VW>(a.w + VW * j, axpy_vec<VW>(scale, sum, ld_vec<VW>(a.w + VW * j)));
+        }
+    }
+    if (blockIdx.x == 0 && threadIdx.x < VW) {
+        const uint64_t i = nv * VW + threadIdx.x;
+        if (i < a.n) {
+            float sum = 0.f;
+            for (uint32_t p = 0; p < P; ++p) sum += ld_stream1(a.grad + (int64_t)p * a.grad_stride + i);
+            const uint32_t reps = REPL ? P : 1;
+            for (uint32_t r = 0; r < reps; ++r) {
+                float *wp = a.w + (int64_t)r * a.w_stride + i;
+                *wp = fmaf(scale, sum, *wp);
+            }
+        }
+    }
+}
+
+// Any 4-byte alignment.
+__global__ void __launch_bounds__(kBlock) static k_dense_sync_scalar(DenseArgs a)
+{
+    pdl_wait_prior_grid();
+    pdl_release_next_grid();
+    const float scale = -a.lr / (float)a.P;
+    const uint64_t stride = (uint64_t)gridDim.x * kBlock;
+    const uint32_t reps = a.w_stride == 0 ? 1 : a.P;
+    for (uint64_t i = (uint64_t)blockIdx.x * kBlock + threadIdx.x; i < a.n; i += stride) {
+        float sum = 0.f;
+        for (uint32_t p = 0; p < a.P; ++p) sum += ld_stream1(a.grad + (int64_t)p * a.grad_stride + i);
+        for (uint32_t r = 0; r < reps; ++r) {
+            float *wp = a.w + (int64_t)r * a.w_stride + i;
+            *wp = fmaf(scale, sum, *wp);
+        }
+    }
+}
+
 // ------------------------------------------------------------------ K4: single cooperative launch
 // For n*P small enough that every thread can keep its share of v in
 // registers: phase 1 loads g (and e) once and reduces, a grid-wide barrier

@@ -432,3 +432,50 @@ def test_bounded_barrier_wait_times_out_cleanly():
     *_, status = B.a2sgd_read_stats(good)
     assert status == B.OK and not torch.equal(w, w0)
     good.destroy()
+
+
+@pytest.mark.parametrize("replicated", [False, True])
+@pytest.mark.parametrize("P,n,pad", [(1, 1, 0), (2, 7, 1), (3, 1000, 0), (4, 65536 + 5, 3), (4, 1 << 20, 0),
+                                     (8, 300_001, 7), (5, 123_456, 0), (16, 4099, 1)])
+def test_dense_sync_step_matches_oracle(replicated, P, n, pad):
+    """Algorithm 1 lines 9-10: the dense averaging step that follows the compressed iterations."""
+    views, raw, stride = _state(4000 + n, P, n, pad=pad, replicated=replicated, g_scale=1e-2)
+    g, e, w = _host(views)
+    ctx = B.a2sgd_create(n, P, 0, EF)
+    B.a2sgd_dense_sync(ctx, views["w"], views["g"], 0.25)
+    torch.cuda.synchronize()
+    oracle.dense_sync(w, g, 0.25)
+    got = views["w"].cpu().numpy()
+    from parity_util import count_outliers, tau_w
+    assert count_outliers(got, w, tau_w(w)) == 0
+    # stricter: an fp32 sum of P terms and one fma against an fp64 reference
+    bound = (P + 2) * np.spacing(np.float32(max(np.abs(w).max(), 0.25 * np.abs(g).max())))
+    assert np.max(np.abs(got.astype(np.float64) - w.astype(np.float64))) <= bound
+    assert np.array_equal(views["g"].cpu().numpy(), g) and np.array_equal(views["e"].cpu().numpy(), e)
+    _guards_intact(raw, views, n, stride, {"g": P, "e": P, "w": P if replicated else 1})
+    ctx.destroy()
+
+
+def test_compressed_iterations_then_dense_sync_like_algorithm_1():
+    """T-1 compressed iterations followed by the dense step, replicas as in Algorithm 1."""
+    wl = W.scaled(W.get_workload("c2_lstm_ptb"), 64)
+    n, P = wl.n, wl.P
+    g = B.padded_rows(P, n, "cuda")
+    w = B.padded_rows(P, n, "cuda")
+    w0 = torch.empty(n, device="cuda")
+    W.init_weights(wl, w0)
+    w.copy_(w0.expand(P, n))
+    w_ref = w.cpu().numpy().copy()
+    ctx = B.a2sgd_create(n, P, 0, ALG1)
+    for step in range(3):
+        W.fill_gradients(wl, step, g)
+        B.a2sgd_step(ctx, w, g, None, wl.lr)
+        lm, gm, cnt, status = B.a2sgd_read_stats(ctx)
+        assert status == B.OK
+        oracle.step(w_ref, g.cpu().numpy(), None, wl.lr, mode=ALG1)
+    W.fill_gradients(wl, 3, g)
+    B.a2sgd_dense_sync(ctx, w, g, wl.lr)
+    oracle.dense_sync(w_ref, g.cpu().numpy(), wl.lr)
+    from parity_util import count_outliers, tau_w
+    assert count_outliers(w.cpu().numpy(), w_ref, tau_w(w_ref)) == 0
+    ctx.destroy()
