@@ -289,6 +289,38 @@ def time_workload(wl, steps, warmup, dev, *, with_roofline=True, with_e2e=True, 
         res["encode_ms"] = enc_ms / k_steps
         res["decode_ms"] = dec_ms / k_steps
 
+    if with_roofline:
+        # rows beyond the core step: the dense synchronisation step (Algorithm 1 lines 9-10) and the
+        # same step over a segment list (one tensor per segment of the workload)
+        k_steps = max(5, min(steps, 50))
+        evs = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+        for _ in range(3):
+            B.a2sgd_dense_sync(ctx, w, g, wl.lr)
+        evs[0].record()
+        for _ in range(k_steps):
+            B.a2sgd_dense_sync(ctx, w, g, wl.lr)
+        evs[1].record()
+        torch.cuda.synchronize(dev)
+        res["dense_sync_ms"] = evs[0].elapsed_time(evs[1]) / k_steps
+        free_b, _ = torch.cuda.mem_get_info(dev)
+        if hasattr(wl, "segments") and free_b > (2 * P + 1) * n * 4 * 1.1:
+            sizes = [sg.numel for sg in wl.segments]
+            gs = [[t.clone() for t in torch.split(g[p], sizes)] for p in range(P)]
+            es = [[t.clone() for t in torch.split(e[p], sizes)] for p in range(P)]
+            ws = [t.clone() for t in torch.split(w, sizes)]
+            plan = B.a2sgd_segments_create(ctx, gs, es, ws)
+            for _ in range(3):
+                B.a2sgd_step_segments(ctx, plan, wl.lr)
+            evs[0].record()
+            for _ in range(k_steps):
+                B.a2sgd_step_segments(ctx, plan, wl.lr)
+            evs[1].record()
+            torch.cuda.synchronize(dev)
+            res["step_segments_ms"] = evs[0].elapsed_time(evs[1]) / k_steps
+            plan.destroy()
+            del gs, es, ws, plan
+            torch.cuda.empty_cache()
+
     if with_e2e:
         try:
             g_host = torch.empty((P, n)).pin_memory()
@@ -473,6 +505,21 @@ def main():
                                        "launch_ms": res["encode_ms"],
                                        "note": "encode + stand-alone global-average launch"}},
     }
+    next_rows = {}
+    if "dense_sync_ms" in res:
+        bts = (4 * wl.P + 8) * wl.n
+        next_rows["dense_sync (Algorithm 1 lines 9-10)"] = {
+            "ms": res["dense_sync_ms"], "GBps": bts / (res["dense_sync_ms"] * 1e-3) / 1e9,
+            "frac_of_measured_peak": bts / (res["dense_sync_ms"] * 1e-3) / 1e9 / peak_gbs,
+            "bytes_per_model_element": 4 * wl.P + 8}
+    if "step_segments_ms" in res:
+        bts = b["step"] * wl.n
+        next_rows["step over a segment list (one tensor per segment)"] = {
+            "ms": res["step_segments_ms"], "GBps": bts / (res["step_segments_ms"] * 1e-3) / 1e9,
+            "frac_of_8TBps": bts / (res["step_segments_ms"] * 1e-3) / 1e9 / NOMINAL_HBM_GBS,
+            "segments": len(wl.segments)}
+    if next_rows:
+        line["next_rows"] = next_rows
     if extra:
         line["other_workloads"] = extra
     if not args.no_cpu_baseline and world == 1:

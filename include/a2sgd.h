@@ -134,6 +134,33 @@ int a2sgd_step(a2sgd_ctx *ctx, float *w, int64_t w_stride,
 int a2sgd_dense_sync(a2sgd_ctx *ctx, float *w, int64_t w_stride,
                      const float *grad, int64_t grad_stride, float lr, void *stream);
 
+/* Segment lists: the model as S separate tensors (the way a training framework holds its
+ * parameters and gradients) instead of one flat vector.  The S tensors are treated as the
+ * concatenation they would form: ONE pair of means per worker over the whole model ("for each
+ * model, it traverses all gradients to compute two separate averages", Section 4.3), the same
+ * results as a2sgd_step on the flattened copy, without making that copy.
+ *
+ * a2sgd_segments_create records the layout once (device tables owned by the plan):
+ *   S           number of tensors; sum of numel[] must equal the context's n
+ *   numel       HOST, [S] element counts (each >= 1)
+ *   grad        HOST array of [P][S] DEVICE pointers, worker-major: grad[p*S + s]
+ *   err         HOST array of [P][S] DEVICE pointers; required in EF mode; in ALG1 mode NULL
+ *               (eps is not stored) or the buffers that receive eps
+ *   w           HOST array of DEVICE pointers: [S] (one shared model) or, when w_replicated
+ *               is non-zero, [P][S] (one replica per worker)
+ * Tensors may have any 4-byte alignment; a tensor all of whose pointers are 32-byte aligned
+ * takes the 256-bit path.  The plan keeps the pointers: the tensors must stay where they are
+ * while the plan is used.  Destroy the plan before its context. */
+typedef struct a2sgd_segments a2sgd_segments;
+int a2sgd_segments_create(a2sgd_ctx *ctx, uint32_t S, const uint64_t *numel,
+                          const float *const *grad, float *const *err, float *const *w,
+                          int w_replicated, a2sgd_segments **out);
+int a2sgd_segments_destroy(a2sgd_segments *plan);
+
+/* One whole loop body of Algorithm 1 (lines 3-7) over a segment list; two launches.  Means and
+ * counts are left in the context for a2sgd_read_stats, as with a2sgd_step. */
+int a2sgd_step_segments(a2sgd_ctx *ctx, a2sgd_segments *plan, float lr, void *stream);
+
 /* a2sgd_step for a caller whose fresh gradients sit in HOST memory (pinned
  * memory makes the copies asynchronous): copies grad_host -> grad_staging
  * worker by worker, runs the step, copies the 2P local and 2 global means

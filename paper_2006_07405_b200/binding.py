@@ -72,6 +72,14 @@ def lib() -> ctypes.CDLL:
                                            _vp, _vp, _vp]
         l.a2sgd_dense_sync.restype = ctypes.c_int
         l.a2sgd_dense_sync.argtypes = [_vp, _vp, _i64, _vp, _i64, ctypes.c_float, _vp]
+        l.a2sgd_segments_create.restype = ctypes.c_int
+        l.a2sgd_segments_create.argtypes = [_vp, ctypes.c_uint32, ctypes.POINTER(ctypes.c_uint64),
+                                            ctypes.POINTER(_vp), ctypes.POINTER(_vp), ctypes.POINTER(_vp),
+                                            ctypes.c_int, ctypes.POINTER(_vp)]
+        l.a2sgd_segments_destroy.restype = ctypes.c_int
+        l.a2sgd_segments_destroy.argtypes = [_vp]
+        l.a2sgd_step_segments.restype = ctypes.c_int
+        l.a2sgd_step_segments.argtypes = [_vp, _vp, ctypes.c_float, _vp]
         l.a2sgd_status_string.restype = ctypes.c_char_p
         l.a2sgd_status_string.argtypes = [ctypes.c_int]
         _lib = l
@@ -217,6 +225,63 @@ def a2sgd_dense_sync(ctx: Context, w: torch.Tensor, grad: torch.Tensor, lr: floa
     wp, ws = _weights(w)
     gp, gs = _rows(grad, "grad")
     _check(lib().a2sgd_dense_sync(ctx.handle, wp, ws, gp, gs, float(lr), _stream(stream)), "a2sgd_dense_sync")
+
+
+class Segments:
+    """Owns an ``a2sgd_segments`` plan and keeps the tensors it points at alive."""
+
+    def __init__(self, ctx: Context, grad, err, w, w_replicated: bool):
+        self.ctx = ctx
+        self._keep = (grad, err, w)
+        P, S = ctx.P, len(grad[0])
+        numel = (ctypes.c_uint64 * S)(*[t.numel() for t in grad[0]])
+
+        def table(rows):
+            flat = [t for row in rows for t in row]
+            for t in flat:
+                if t.dtype != torch.float32 or not t.is_cuda or not t.is_contiguous():
+                    raise ValueError("segments: need contiguous float32 CUDA tensors")
+            return (_vp * len(flat))(*[t.data_ptr() for t in flat])
+
+        if len(grad) != P or any(len(r) != S for r in grad):
+            raise ValueError("grad: need P lists of S tensors")
+        g_tab = table(grad)
+        e_tab = table(err) if err is not None else None
+        w_tab = table(w if w_replicated else [w])
+        self._h = _vp()
+        _check(lib().a2sgd_segments_create(ctx.handle, S, numel, g_tab, e_tab, w_tab, 1 if w_replicated else 0,
+                                           ctypes.byref(self._h)), "a2sgd_segments_create")
+
+    @property
+    def handle(self):
+        if not self._h:
+            raise RuntimeError("segment plan destroyed")
+        return self._h
+
+    def destroy(self) -> None:
+        if self._h:
+            lib().a2sgd_segments_destroy(self._h)
+            self._h = _vp()
+
+    def __del__(self):
+        try:
+            self.destroy()
+        except Exception:
+            pass
+
+
+def a2sgd_segments_create(ctx: Context, grad, err, w, w_replicated: bool = False) -> Segments:
+    """grad / err: P lists of S tensors (err None in ALG1 mode when eps is not wanted);
+    w: a list of S tensors (shared) or P lists of S tensors (replicated)."""
+    return Segments(ctx, grad, err, w, w_replicated)
+
+
+def a2sgd_segments_destroy(plan: Segments) -> None:
+    plan.destroy()
+
+
+def a2sgd_step_segments(ctx: Context, plan: Segments, lr: float, stream=None) -> None:
+    _check(lib().a2sgd_step_segments(ctx.handle, plan.handle, float(lr), _stream(stream)), "a2sgd_step_segments")
 
 
 def a2sgd_step_host(ctx: Context, w: torch.Tensor, grad_host: torch.Tensor, grad_staging: torch.Tensor,

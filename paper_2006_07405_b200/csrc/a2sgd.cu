@@ -8,8 +8,10 @@
 #include <cstdint>
 #include <new>
 #include <unordered_map>
+#include <vector>
 
 #include "a2sgd_kernels.cuh"
+#include "a2sgd_segments.cuh"
 
 using namespace a2sgd;
 
@@ -50,6 +52,20 @@ struct a2sgd_ctx {
     unsigned int coop_epoch = 0;
     // resident CTAs per SM of every kernel instance used so far (occupancy API, cached)
     std::unordered_map<const void *, int> occ;
+};
+
+struct a2sgd_segments {
+    a2sgd_ctx *ctx = nullptr;
+    uint32_t S = 0;
+    bool replicated = false;
+    bool has_err = false;
+    // device tables
+    SegTile *tiles = nullptr;
+    uint64_t n_tiles = 0;
+    uint64_t *numel = nullptr;
+    const float **grad = nullptr;
+    float **err = nullptr;
+    float **w = nullptr;
 };
 
 namespace {
@@ -548,6 +564,135 @@ extern "C" int a2sgd_dense_sync(a2sgd_ctx *c, float *w, int64_t w_stride, const 
     const dim3 grid(flat_grid(c, occupancy(c, fn), items, A2SGD_WAVES_K3));
     void *params[] = {&a};
     A2_CUDA(launch_pdl(fn, grid, params, static_cast<cudaStream_t>(stream)));
+    return A2SGD_OK;
+}
+
+// ---------------------------------------------------------------- segment lists
+template <bool EF, bool STORE>
+const void *select_decode_segments_p(uint32_t P)
+{
+    switch (P) {
+    case 1: return (const void *)k_decode_segments<EF, STORE, 1>;
+    case 2: return (const void *)k_decode_segments<EF, STORE, 2>;
+    case 4: return (const void *)k_decode_segments<EF, STORE, 4>;
+    case 8: return (const void *)k_decode_segments<EF, STORE, 8>;
+    default: return (const void *)k_decode_segments<EF, STORE, 0>;
+    }
+}
+
+extern "C" int a2sgd_segments_create(a2sgd_ctx *c, uint32_t S, const uint64_t *numel, const float *const *grad,
+                                     float *const *err, float *const *w, int w_replicated, a2sgd_segments **out)
+{
+    if (!out) return A2SGD_ERR_ARG;
+    *out = nullptr;
+    if (!c || S == 0 || !numel || !grad || !w) return A2SGD_ERR_ARG;
+    if (!c->alg1 && !err) return A2SGD_ERR_ARG;
+    const uint32_t P = c->P;
+    const bool repl = w_replicated != 0 && P > 1;
+    uint64_t total = 0;
+    std::vector<SegTile> tiles;
+    for (uint32_t s = 0; s < S; ++s) {
+        if (numel[s] == 0) return A2SGD_ERR_ARG;
+        total += numel[s];
+        bool vec = true;
+        for (uint32_t p = 0; p < P; ++p) {
+            const float *g = grad[(size_t)p * S + s];
+            const float *e = err ? err[(size_t)p * S + s] : nullptr;
+            if (!g || (!c->alg1 && !e)) return A2SGD_ERR_ARG;
+            if (!aligned(g, 4) || (e && !aligned(e, 4))) return A2SGD_ERR_ALIGN;
+            vec = vec && aligned(g, 32) && (!e || aligned(e, 32));
+        }
+        const uint32_t w_rows = repl ? P : 1;
+        for (uint32_t r = 0; r < w_rows; ++r) {
+            const float *wp = w[(size_t)r * S + s];
+            if (!wp) return A2SGD_ERR_ARG;
+            if (!aligned(wp, 4)) return A2SGD_ERR_ALIGN;
+            vec = vec && aligned(wp, 32);
+        }
+        for (uint64_t off = 0; off < numel[s]; off += kSegTile) tiles.push_back(SegTile{s, vec ? kSegFlagVec : 0u, off});
+    }
+    if (total != c->n) return A2SGD_ERR_ARG;
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return A2SGD_ERR_CUDA;
+    a2sgd_segments *sg = new (std::nothrow) a2sgd_segments();
+    if (!sg) return A2SGD_ERR_NOMEM;
+    sg->ctx = c;
+    sg->S = S;
+    sg->replicated = repl;
+    sg->has_err = err != nullptr;
+    sg->n_tiles = tiles.size();
+    const size_t w_count = (size_t)(repl ? P : 1) * S;
+    bool ok = true;
+    ok = ok && cudaMalloc(&sg->tiles, sizeof(SegTile) * tiles.size()) == cudaSuccess;
+    ok = ok && cudaMalloc(&sg->numel, sizeof(uint64_t) * S) == cudaSuccess;
+    ok = ok && cudaMalloc(&sg->grad, sizeof(float *) * (size_t)P * S) == cudaSuccess;
+    ok = ok && cudaMalloc(&sg->w, sizeof(float *) * w_count) == cudaSuccess;
+    if (err) ok = ok && cudaMalloc(&sg->err, sizeof(float *) * (size_t)P * S) == cudaSuccess;
+    ok = ok && cudaMemcpy(sg->tiles, tiles.data(), sizeof(SegTile) * tiles.size(), cudaMemcpyHostToDevice) == cudaSuccess;
+    ok = ok && cudaMemcpy(sg->numel, numel, sizeof(uint64_t) * S, cudaMemcpyHostToDevice) == cudaSuccess;
+    ok = ok && cudaMemcpy(sg->grad, grad, sizeof(float *) * (size_t)P * S, cudaMemcpyHostToDevice) == cudaSuccess;
+    ok = ok && cudaMemcpy(sg->w, w, sizeof(float *) * w_count, cudaMemcpyHostToDevice) == cudaSuccess;
+    if (err) ok = ok && cudaMemcpy(sg->err, err, sizeof(float *) * (size_t)P * S, cudaMemcpyHostToDevice) == cudaSuccess;
+    if (!ok) {
+        (void)cudaGetLastError();
+        a2sgd_segments_destroy(sg);
+        return A2SGD_ERR_NOMEM;
+    }
+    *out = sg;
+    return A2SGD_OK;
+}
+
+extern "C" int a2sgd_segments_destroy(a2sgd_segments *sg)
+{
+    if (!sg) return A2SGD_OK;
+    DeviceGuard guard(sg->ctx->device);
+    cudaFree(sg->tiles);
+    cudaFree(sg->numel);
+    cudaFree(sg->grad);
+    cudaFree(sg->err);
+    cudaFree(sg->w);
+    (void)cudaGetLastError();
+    delete sg;
+    return A2SGD_OK;
+}
+
+extern "C" int a2sgd_step_segments(a2sgd_ctx *c, a2sgd_segments *sg, float lr, void *stream)
+{
+    if (!c || !sg || sg->ctx != c) return A2SGD_ERR_ARG;
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return A2SGD_ERR_CUDA;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const bool ef = !c->alg1;
+    const bool store = ef || sg->has_err;
+    SegTables t{};
+    t.tiles = sg->tiles;
+    t.n_tiles = sg->n_tiles;
+    t.numel = sg->numel;
+    t.grad = sg->grad;
+    t.err = sg->err;
+    t.w = sg->w;
+    t.S = sg->S;
+    t.w_replicated = sg->replicated ? 1u : 0u;
+    {
+        EncodeArgs a = make_encode_args(c, nullptr, 0, nullptr, 0, c->local_means, c->pos_counts, nullptr,
+                                        c->global_means);
+        const void *fn = ef ? (const void *)k_encode_segments<true> : (const void *)k_encode_segments<false>;
+        const uint64_t slots = (uint64_t)c->sm_count * occupancy(c, fn) * A2SGD_WAVES_K1;
+        uint64_t G = std::max<uint64_t>(1, slots / c->P);
+        G = std::min<uint64_t>(std::min<uint64_t>(G, sg->n_tiles), c->g_alloc);
+        void *params[] = {&a, &t};
+        A2_CUDA(launch_pdl(fn, dim3((unsigned)G, c->P), params, s));
+    }
+    {
+        DecodeArgs a = make_decode_args(c, nullptr, sg->replicated ? 1 : 0, nullptr, 0, nullptr, 0, c->local_means,
+                                        c->global_means, lr);
+        const void *fn = ef ? select_decode_segments_p<true, true>(c->P)
+                            : store ? select_decode_segments_p<false, true>(c->P)
+                                    : select_decode_segments_p<false, false>(c->P);
+        const uint64_t grid = std::min<uint64_t>(sg->n_tiles, 0x7fffffffu);
+        void *params[] = {&a, &t};
+        A2_CUDA(launch_pdl(fn, dim3((unsigned)grid), params, s));
+    }
     return A2SGD_OK;
 }
 

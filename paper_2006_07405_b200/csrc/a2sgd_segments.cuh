@@ -1,0 +1,196 @@
+// Segment-list (multi-tensor) forms of K1 and K3: the model is a list of
+// tensors living in separate allocations, as a training framework holds them,
+// and is reduced to the same two whole-model means per worker ("for each
+// model, it traverses all gradients to compute two separate averages",
+// Section 4.3) without first being copied into one flat vector.
+//
+// The flat index space of each tensor is cut into tiles of kSegTile elements;
+// a table built once per plan maps tile -> (tensor, offset).  A tile never
+// crosses a tensor boundary, so all addressing inside a tile is one base
+// pointer plus a contiguous range.  Tensors whose pointers are all 32-byte
+// aligned take 256-bit accesses; any other 4-byte alignment takes coalesced
+// scalar accesses (decided per tensor on the host, uniform per CTA).
+#pragma once
+
+#include "a2sgd_kernels.cuh"
+
+namespace a2sgd {
+
+constexpr int kSegVW = 8;
+constexpr uint32_t kSegTile = kBlock * kSegVW; // 2048 elements per tile
+constexpr uint32_t kSegFlagVec = 1u;
+
+struct __align__(16) SegTile {
+    uint32_t seg;    // tensor index
+    uint32_t flags;  // kSegFlagVec: every pointer of this tensor is 32-byte aligned
+    uint64_t offset; // first element of the tile inside the tensor
+};
+
+struct SegTables {
+    const SegTile *tiles;
+    uint64_t n_tiles;
+    const uint64_t *numel;      // [S]
+    const float *const *grad;   // [P][S] device pointers, worker-major
+    float *const *err;          // [P][S] or nullptr
+    float *const *w;            // [S] (shared) or [P][S] (replicas)
+    uint32_t S;
+    uint32_t w_replicated;
+};
+
+// K1 over a segment list.  grid = (G, P); CTA x walks tiles x, x + G, ...
+template <bool EF>
+__global__ void __launch_bounds__(kBlock) k_encode_segments(EncodeArgs a, SegTables t)
+{
+    pdl_wait_prior_grid();
+    pdl_release_next_grid();
+    __shared__ double sh_d[2][kWarps];
+    __shared__ unsigned long long sh_n[kWarps];
+    __shared__ int sh_flag;
+    const uint32_t p = blockIdx.y;
+    Acc acc;
+    for (uint64_t tile = blockIdx.x; tile < t.n_tiles; tile += gridDim.x) {
+        const SegTile d = t.tiles[tile];
+        const uint64_t n_s = t.numel[d.seg];
+        const float *__restrict__ g = t.grad[(uint64_t)p * t.S + d.seg];
+        const float *__restrict__ e = EF ? t.err[(uint64_t)p * t.S + d.seg] : nullptr;
+        float sp = 0.f, sn = 0.f;
+        unsigned bits;
+        const uint64_t i = d.offset + (uint64_t)threadIdx.x * kSegVW;
+        if ((d.flags & kSegFlagVec) && i + kSegVW <= n_s) {
+            Vec<kSegVW> v = ld_vec<kSegVW>(g + i);
+            if (EF) v = add_vec<kSegVW>(v, ld_vec<kSegVW>(e + i));
+            split_vec<kSegVW>(v, sp, sn, acc.n_pos, bits);
+        } else if (d.flags & kSegFlagVec) {
+            // the tensor's last, partial vector
+            float ps[kSegVW], ns[kSegVW];
+#pragma unroll
+            for (int k = 0; k < kSegVW; ++k) {
+                ps[k] = ns[k] = 0.f;
+                if (i + k < n_s) {
+                    float v = ld_stream1(g + i + k);
+                    if (EF) v += ld_stream1(e + i + k);
+                    unsigned b;
+                    split1(v, ps[k], ns[k], acc.n_pos, b);
+                }
+            }
+            sp = tree_sum<kSegVW>(ps);
+            sn = tree_sum<kSegVW>(ns);
+        } else {
+            float ps[kSegVW], ns[kSegVW];
+#pragma unroll
+            for (int k = 0; k < kSegVW; ++k) {
+                const uint64_t idx = d.offset + (uint64_t)k * kBlock + threadIdx.x;
+                ps[k] = ns[k] = 0.f;
+                if (idx < n_s) {
+                    float v = ld_stream1(g + idx);
+                    if (EF) v += ld_stream1(e + idx);
+                    unsigned b;
+                    split1(v, ps[k], ns[k], acc.n_pos, b);
+                }
+            }
+            sp = tree_sum<kSegVW>(ps);
+            sn = tree_sum<kSegVW>(ns);
+        }
+        acc.s_pos += (double)sp;
+        acc.s_neg += (double)sn;
+    }
+    double s_pos = acc.s_pos, s_neg = acc.s_neg;
+    unsigned long long n_pos = acc.n_pos;
+    block_reduce(s_pos, s_neg, n_pos, sh_d, sh_n);
+    finish_worker(a, p, s_pos, s_neg, n_pos, sh_d, sh_n, &sh_flag);
+}
+
+// K3 over a segment list: one tile per CTA.  PT > 0: compile-time worker count.
+template <bool EF, bool STORE, int PT>
+__global__ void __launch_bounds__(kBlock) k_decode_segments(DecodeArgs a, SegTables t)
+{
+    pdl_wait_prior_grid();
+    pdl_release_next_grid();
+    __shared__ WorkerConst sh_c[PT > 0 ? 1 : kMaxP];
+    const uint32_t P = PT > 0 ? PT : a.P;
+    const float m_pos = __ldg(a.global_means), m_neg = __ldg(a.global_means + 1);
+    const bool repl = t.w_replicated != 0;
+    const float scale = repl ? -a.lr : -a.lr / (float)P;
+    if (PT == 0) {
+        for (uint32_t p = threadIdx.x; p < P; p += kBlock) sh_c[p] = worker_const<EF>(a, p, m_pos, m_neg);
+        __syncthreads();
+    }
+    for (uint64_t tile = blockIdx.x; tile < t.n_tiles; tile += gridDim.x) {
+        const SegTile d = t.tiles[tile];
+        const uint64_t n_s = t.numel[d.seg];
+        const uint64_t i = d.offset + (uint64_t)threadIdx.x * kSegVW;
+        if ((d.flags & kSegFlagVec) && i + kSegVW <= n_s) {
+            if (PT > 0 && !repl) {
+                constexpr int PP = PT > 0 ? PT : 1;
+                Vec<kSegVW> gv[PP], ev[PP];
+                float *wp = t.w[d.seg] + i;
+                const Vec<kSegVW> wv = ld_vec<kSegVW>(wp);
+#pragma unroll
+                for (int p = 0; p < PP; ++p) gv[p] = ld_vec<kSegVW>(t.grad[(uint64_t)p * t.S + d.seg] + i);
+                if (EF) {
+#pragma unroll
+                    for (int p = 0; p < PP; ++p) ev[p] = ld_vec<kSegVW>(t.err[(uint64_t)p * t.S + d.seg] + i);
+                }
+                Vec<kSegVW> sum = zero_vec<kSegVW>();
+#pragma unroll
+                for (int p = 0; p < PP; ++p) {
+                    const Vec<kSegVW> v = EF ? add_vec<kSegVW>(gv[p], ev[p]) : gv[p];
+                    Vec<kSegVW> gh, rs;
+                    decode_vec<EF, kSegVW>(v, worker_const<EF>(a, p, m_pos, m_neg), gh, rs);
+                    sum = add_vec<kSegVW>(sum, gh);
+                    if (STORE) st_vec<kSegVW>(t.err[(uint64_t)p * t.S + d.seg] + i, rs);
+                }
+                st_vec<kSegVW>(wp, axpy_vec<kSegVW>(scale, sum, wv));
+            } else {
+                Vec<kSegVW> sum = zero_vec<kSegVW>();
+                for (uint32_t p = 0; p < P; ++p) {
+                    const WorkerConst c = PT > 0 ? worker_const<EF>(a, p, m_pos, m_neg) : sh_c[p];
+                    Vec<kSegVW> v = ld_vec<kSegVW>(t.grad[(uint64_t)p * t.S + d.seg] + i);
+                    if (EF) v = add_vec<kSegVW>(v, ld_vec<kSegVW>(t.err[(uint64_t)p * t.S + d.seg] + i));
+                    Vec<kSegVW> gh, rs;
+                    decode_vec<EF, kSegVW>(v, c, gh, rs);
+                    if (STORE) st_vec<kSegVW>(t.err[(uint64_t)p * t.S + d.seg] + i, rs);
+                    if (repl) {
+                        float *wp = t.w[(uint64_t)p * t.S + d.seg] + i;
+                        st_vec<kSegVW>(wp, axpy_vec<kSegVW>(scale, gh, ld_vec<kSegVW>(wp)));
+                    } else {
+                        sum = add_vec<kSegVW>(sum, gh);
+                    }
+                }
+                if (!repl) {
+                    float *wp = t.w[d.seg] + i;
+                    st_vec<kSegVW>(wp, axpy_vec<kSegVW>(scale, sum, ld_vec<kSegVW>(wp)));
+                }
+            }
+        } else {
+            // scalar elements: a misaligned tensor (coalesced, stride kBlock) or a tensor's last partial vector
+            const bool vec_tail = (d.flags & kSegFlagVec) != 0;
+#pragma unroll 1
+            for (int k = 0; k < kSegVW; ++k) {
+                const uint64_t idx = vec_tail ? i + k : d.offset + (uint64_t)k * kBlock + threadIdx.x;
+                if (idx >= n_s) continue;
+                float sum = 0.f;
+                for (uint32_t p = 0; p < P; ++p) {
+                    const WorkerConst c = PT > 0 ? worker_const<EF>(a, p, m_pos, m_neg) : sh_c[p];
+                    float v = ld_stream1(t.grad[(uint64_t)p * t.S + d.seg] + idx);
+                    if (EF) v += ld_stream1(t.err[(uint64_t)p * t.S + d.seg] + idx);
+                    float gh, rs;
+                    decode1<EF>(v, c, gh, rs);
+                    if (STORE) st_stream1(t.err[(uint64_t)p * t.S + d.seg] + idx, rs);
+                    if (repl) {
+                        float *wp = t.w[(uint64_t)p * t.S + d.seg] + idx;
+                        *wp = fmaf(scale, gh, *wp);
+                    } else {
+                        sum += gh;
+                    }
+                }
+                if (!repl) {
+                    float *wp = t.w[d.seg] + idx;
+                    *wp = fmaf(scale, sum, *wp);
+                }
+            }
+        }
+    }
+}
+
+} // namespace a2sgd

@@ -1,0 +1,115 @@
+"""Segment-list entry points: the model as separate tensors (any alignment), reduced to the same
+whole-model means as the flat path.  Reference: the CPU oracle on the concatenation."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2006_07405_b200 import binding as B
+from paper_2006_07405_b200 import workloads as W
+from parity_util import assert_means, assert_state
+
+pytestmark = pytest.mark.gpu
+EF, ALG1 = B.MODE_EF, B.MODE_ALG1
+
+
+def _tensors(sizes, offsets, gen, scale):
+    """One tensor per size; tensor k starts offsets[k % len(offsets)] elements into its own allocation."""
+    out = []
+    for k, n in enumerate(sizes):
+        o = offsets[k % len(offsets)]
+        buf = torch.full((n + o + 8,), float("nan"), device="cuda")
+        t = buf[o:o + n]
+        t.normal_(0.0, scale, generator=gen)
+        out.append(t)
+    return out
+
+
+def _cat(rows):
+    return np.stack([torch.cat(r).cpu().numpy() for r in rows])
+
+
+@pytest.mark.parametrize("mode", [EF, ALG1])
+@pytest.mark.parametrize("replicated", [False, True])
+@pytest.mark.parametrize("P,offsets", [(1, [0]), (4, [0]), (3, [0, 1, 0, 8, 3]), (8, [0, 0, 0, 2]), (2, [1])])
+def test_segment_list_step_matches_oracle_on_concatenation(mode, replicated, P, offsets):
+    wl = W.scaled(W.get_workload("c3_resnet50"), 16)        # 161 tensors, many of them tiny
+    sizes = [s.numel for s in wl.segments] + [1, 2, 7, 2047, 2048, 2049, 4096 + 8]
+    n = sum(sizes)
+    gen = torch.Generator("cuda").manual_seed(P * 100 + len(offsets))
+    grad = [_tensors(sizes, offsets, gen, 1e-3) for _ in range(P)]
+    err = [_tensors(sizes, offsets, gen, 3e-4) for _ in range(P)]
+    w = [_tensors(sizes, offsets, gen, 0.02) for _ in range(P if replicated else 1)]
+    gh, eh = _cat(grad), _cat(err)
+    wh = _cat(w) if replicated else _cat(w)[0]
+    ctx = B.a2sgd_create(n, P, 0, mode)
+    plan = B.a2sgd_segments_create(ctx, grad, err, w if replicated else w[0], w_replicated=replicated)
+    B.a2sgd_step_segments(ctx, plan, 0.1)
+    lm, gm, cnt, status = B.a2sgd_read_stats(ctx)
+    lm_ref, gm_ref, cnt_ref = oracle.step(wh, gh, eh, 0.1, mode=mode)
+    assert status == B.OK and np.array_equal(cnt, cnt_ref)
+    assert_means(lm, lm_ref)
+    assert_means(gm, gm_ref)
+    w_got = _cat(w) if replicated else _cat(w)[0]
+    assert_state(w_got, wh, _cat(err), eh, gm_ref, f"segments P={P}")
+    assert np.array_equal(_cat(grad), gh)                    # gradients untouched
+    for rows in (grad, err, w):                              # nothing written outside the tensors
+        for row in rows:
+            for t in row:
+                base = t.untyped_storage()
+                full = torch.tensor([], dtype=torch.float32, device="cuda").set_(base)
+                o = t.storage_offset()
+                assert torch.isnan(full[:o]).all() and torch.isnan(full[o + t.numel():]).all()
+    plan.destroy()
+    ctx.destroy()
+
+
+def test_segment_list_equals_flat_path_and_is_reproducible():
+    wl = W.scaled(W.get_workload("c2_lstm_ptb"), 32)
+    n, P = wl.n, wl.P
+    flat_g = B.padded_rows(P, n, "cuda")
+    W.fill_gradients(wl, 0, flat_g)
+    flat_e = B.padded_rows(P, n, "cuda", fill=0.0)
+    flat_w = torch.empty(n, device="cuda")
+    W.init_weights(wl, flat_w)
+    sizes = [s.numel for s in wl.segments]
+
+    def split(row):
+        return [t.clone() for t in torch.split(row, sizes)]
+
+    outs = []
+    for _ in range(2):
+        grad = [split(flat_g[p]) for p in range(P)]
+        err = [split(flat_e[p]) for p in range(P)]
+        w = split(flat_w)
+        ctx = B.a2sgd_create(n, P, 0, EF)
+        plan = B.a2sgd_segments_create(ctx, grad, err, w)
+        B.a2sgd_step_segments(ctx, plan, wl.lr)
+        lm, gm, cnt, status = B.a2sgd_read_stats(ctx)
+        outs.append((lm.tobytes(), gm.tobytes(), cnt.tobytes(), torch.cat(w).cpu().numpy().tobytes(),
+                     _cat(err).tobytes()))
+        plan.destroy()
+        ctx.destroy()
+    assert outs[0] == outs[1]
+    ctx = B.a2sgd_create(n, P, 0, EF | B.FORCE_TWO_PASS)
+    B.a2sgd_step(ctx, flat_w, flat_g, flat_e, wl.lr)
+    lm_f, gm_f, cnt_f, _ = B.a2sgd_read_stats(ctx)
+    assert np.array_equal(cnt_f, cnt)
+    assert_means(lm, lm_f)
+    assert_means(gm, gm_f)
+    assert_state(torch.cat(w).cpu().numpy(), flat_w.cpu().numpy(), _cat(err), flat_e.cpu().numpy(), gm_f, "flat vs segments")
+    ctx.destroy()
+
+
+def test_segment_plan_argument_checks():
+    ctx = B.a2sgd_create(100, 2, 0, EF)
+    g = [[torch.zeros(60, device="cuda"), torch.zeros(40, device="cuda")] for _ in range(2)]
+    w = [torch.zeros(60, device="cuda"), torch.zeros(40, device="cuda")]
+    with pytest.raises(B.A2SGDError) as ei:
+        B.a2sgd_segments_create(ctx, g, None, w)                 # EF needs err
+    assert ei.value.status == B.ERR_ARG
+    bad = [[torch.zeros(60, device="cuda"), torch.zeros(41, device="cuda")] for _ in range(2)]
+    with pytest.raises(B.A2SGDError) as ei:
+        B.a2sgd_segments_create(ctx, bad, bad, w)                # sizes do not add up to n
+    assert ei.value.status == B.ERR_ARG
+    ctx.destroy()
