@@ -568,22 +568,30 @@ __global__ void __launch_bounds__(kBlock) k_decode_shared_vec(DecodeArgs a)
 #pragma unroll
         for (int p = 0; p < PP; ++p) c[p] = worker_const<EF>(a, p, m_pos, m_neg);
         for (uint64_t j = (uint64_t)blockIdx.x * kBlock + threadIdx.x; j < nv; j += stride) {
-            Vec<VW> gv[PP], ev[PP];
+            // workers whose loads are in flight together; 4 measured better than 8 at P = 8
+            // (6.55 -> 6.77 TB/s): fewer concurrent streams per thread, lower register count
+            constexpr int PB = PP < 4 ? PP : 4;
             const Vec<VW> wv = ld_vec<VW>(a.w + VW * j);
-#pragma unroll
-            for (int p = 0; p < PP; ++p) gv[p] = ld_vec<VW>(a.grad + (int64_t)p * a.grad_stride + VW * j);
-            if (EF) {
-#pragma unroll
-                for (int p = 0; p < PP; ++p) ev[p] = ld_vec<VW>(a.err + (int64_t)p * a.err_stride + VW * j);
-            }
             Vec<VW> sum = zero_vec<VW>();
 #pragma unroll
-            for (int p = 0; p < PP; ++p) {
-                const Vec<VW> v = EF ? add_vec<VW>(gv[p], ev[p]) : gv[p];
-                Vec<VW> gh, rs;
-                decode_vec<EF, VW>(v, c[p], gh, rs);
-                sum = add_vec<VW>(sum, gh);
-                if (STORE) st_vec<VW>(a.err + (int64_t)p * a.err_stride + VW * j, rs);
+            for (int p0 = 0; p0 < PP; p0 += PB) {
+                Vec<VW> gv[PB], ev[PB];
+#pragma unroll
+                for (int q = 0; q < PB; ++q)
+                    gv[q] = ld_vec<VW>(a.grad + (int64_t)(p0 + q) * a.grad_stride + VW * j);
+                if (EF) {
+#pragma unroll
+                    for (int q = 0; q < PB; ++q)
+                        ev[q] = ld_vec<VW>(a.err + (int64_t)(p0 + q) * a.err_stride + VW * j);
+                }
+#pragma unroll
+                for (int q = 0; q < PB; ++q) {
+                    const Vec<VW> v = EF ? add_vec<VW>(gv[q], ev[q]) : gv[q];
+                    Vec<VW> gh, rs;
+                    decode_vec<EF, VW>(v, c[p0 + q], gh, rs);
+                    sum = add_vec<VW>(sum, gh);
+                    if (STORE) st_vec<VW>(a.err + (int64_t)(p0 + q) * a.err_stride + VW * j, rs);
+                }
             }
             st_vec<VW>(a.w + VW * j, axpy_vec<VW>(scale, sum, wv));
         }
