@@ -302,6 +302,17 @@ def time_workload(wl, steps, warmup, dev, *, with_roofline=True, with_e2e=True, 
         evs[1].record()
         torch.cuda.synchronize(dev)
         res["dense_sync_ms"] = evs[0].elapsed_time(evs[1]) / k_steps
+        g16 = torch.empty((P, g.stride(0)), dtype=torch.bfloat16, device=dev)[:, :n]
+        g16.copy_(g)
+        for _ in range(3):
+            B.a2sgd_step_bf16(ctx, w, g16, e, wl.lr)
+        evs[0].record()
+        for _ in range(k_steps):
+            B.a2sgd_step_bf16(ctx, w, g16, e, wl.lr)
+        evs[1].record()
+        torch.cuda.synchronize(dev)
+        res["step_bf16_ms"] = evs[0].elapsed_time(evs[1]) / k_steps
+        del g16
         free_b, _ = torch.cuda.mem_get_info(dev)
         if hasattr(wl, "segments") and free_b > (2 * P + 1) * n * 4 * 1.1:
             sizes = [sg.numel for sg in wl.segments]
@@ -518,6 +529,12 @@ def main():
             "ms": res["step_segments_ms"], "GBps": bts / (res["step_segments_ms"] * 1e-3) / 1e9,
             "frac_of_8TBps": bts / (res["step_segments_ms"] * 1e-3) / 1e9 / NOMINAL_HBM_GBS,
             "segments": len(wl.segments)}
+    if "step_bf16_ms" in res:
+        bts = (16 * wl.P + 8) * wl.n
+        next_rows["step with bfloat16 gradients"] = {
+            "ms": res["step_bf16_ms"], "GBps": bts / (res["step_bf16_ms"] * 1e-3) / 1e9,
+            "frac_of_8TBps": bts / (res["step_bf16_ms"] * 1e-3) / 1e9 / NOMINAL_HBM_GBS,
+            "model_params_per_s": wl.n / (res["step_bf16_ms"] * 1e-3), "bytes_per_model_element": 16 * wl.P + 8}
     if next_rows:
         line["next_rows"] = next_rows
     if extra:

@@ -125,6 +125,18 @@ int a2sgd_step(a2sgd_ctx *ctx, float *w, int64_t w_stride,
                const float *grad, int64_t grad_stride,
                float *err, int64_t err_stride, float lr, void *stream);
 
+/* a2sgd_step with the fresh gradients stored as bfloat16 (the paper remarks that the method
+ * "can be further integrated with quantization"; a bfloat16 gradient is the common case of a
+ * mixed-precision backward pass).  grad: [P] vectors of n bfloat16 values (raw uint16 bit
+ * patterns), worker stride grad_stride in ELEMENTS.  Widening bfloat16 to fp32 is exact, so the
+ * result equals a2sgd_step on the widened gradients; err and w stay fp32.  Traffic drops from
+ * (20P + 8) to (16P + 8) bytes per model element.  Always two launches.  The fast path needs
+ * 16-byte aligned gradient rows with strides that are multiples of 8 elements and 32-byte
+ * aligned err / w rows; anything else takes the scalar kernels. */
+int a2sgd_step_bf16(a2sgd_ctx *ctx, float *w, int64_t w_stride,
+                    const uint16_t *grad, int64_t grad_stride,
+                    float *err, int64_t err_stride, float lr, void *stream);
+
 /* Algorithm 1 lines 9-10: the dense synchronisation that follows the last compressed iteration
  * (Eq. 1 for one step).  The workers' gradients are averaged element-wise, summed in worker
  * order, and applied: w <- w - lr * (1/P) * sum_p grad^p.  With w_stride == 0 the one shared w is

@@ -80,6 +80,8 @@ def lib() -> ctypes.CDLL:
         l.a2sgd_segments_destroy.argtypes = [_vp]
         l.a2sgd_step_segments.restype = ctypes.c_int
         l.a2sgd_step_segments.argtypes = [_vp, _vp, ctypes.c_float, _vp]
+        l.a2sgd_step_bf16.restype = ctypes.c_int
+        l.a2sgd_step_bf16.argtypes = [_vp, _vp, _i64, _vp, _i64, _vp, _i64, ctypes.c_float, _vp]
         l.a2sgd_status_string.restype = ctypes.c_char_p
         l.a2sgd_status_string.argtypes = [ctypes.c_int]
         _lib = l
@@ -218,6 +220,17 @@ def a2sgd_step(ctx: Context, w: torch.Tensor, grad: torch.Tensor, err: Optional[
     gp, gs = _rows(grad, "grad")
     ep, es = _rows(err, "err")
     _check(lib().a2sgd_step(ctx.handle, wp, ws, gp, gs, ep, es, float(lr), _stream(stream)), "a2sgd_step")
+
+
+def a2sgd_step_bf16(ctx: Context, w: torch.Tensor, grad: torch.Tensor, err: Optional[torch.Tensor], lr: float,
+                    stream=None) -> None:
+    """a2sgd_step with bfloat16 gradients: grad is a torch.bfloat16 CUDA tensor [P, >= n]."""
+    if grad.dtype != torch.bfloat16 or not grad.is_cuda or grad.dim() != 2 or (grad.shape[1] > 1 and grad.stride(1) != 1):
+        raise ValueError("grad: need a bfloat16 CUDA tensor [P, n] with unit inner stride")
+    wp, ws = _weights(w)
+    ep, es = _rows(err, "err")
+    _check(lib().a2sgd_step_bf16(ctx.handle, wp, ws, grad.data_ptr(), grad.stride(0), ep, es, float(lr),
+                                 _stream(stream)), "a2sgd_step_bf16")
 
 
 def a2sgd_dense_sync(ctx: Context, w: torch.Tensor, grad: torch.Tensor, lr: float, stream=None) -> None:

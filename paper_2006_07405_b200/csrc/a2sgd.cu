@@ -210,6 +210,45 @@ const void *select_decode_scalar(bool ef, bool store)
     return store ? (const void *)k_decode_scalar<false, true> : (const void *)k_decode_scalar<false, false>;
 }
 
+// bfloat16 gradient rows: 8-element (128-bit) vectors or scalar accesses
+template <bool EF, bool STORE>
+const void *select_decode_shared_bf16_p(uint32_t P)
+{
+    switch (P) {
+    case 1: return (const void *)k_decode_shared_vec<EF, STORE, 1, 8, true>;
+    case 2: return (const void *)k_decode_shared_vec<EF, STORE, 2, 8, true>;
+    case 4: return (const void *)k_decode_shared_vec<EF, STORE, 4, 8, true>;
+    case 8: return (const void *)k_decode_shared_vec<EF, STORE, 8, 8, true>;
+    default: return (const void *)k_decode_shared_vec<EF, STORE, 0, 8, true>;
+    }
+}
+
+const void *select_encode_bf16(bool ef, int vw)
+{
+    if (vw == 8) return ef ? (const void *)k_encode_vec<true, false, 8, true> : (const void *)k_encode_vec<false, false, 8, true>;
+    return ef ? (const void *)k_encode_scalar<true, false, true> : (const void *)k_encode_scalar<false, false, true>;
+}
+
+const void *select_decode_bf16(bool ef, bool store, bool shared, uint32_t P, int vw)
+{
+    if (vw == 8 && shared) {
+        if (ef) return select_decode_shared_bf16_p<true, true>(P);
+        return store ? select_decode_shared_bf16_p<false, true>(P) : select_decode_shared_bf16_p<false, false>(P);
+    }
+    if (vw == 8) {
+        if (ef) return (const void *)k_decode_repl_vec<true, true, 8, true>;
+        return store ? (const void *)k_decode_repl_vec<false, true, 8, true> : (const void *)k_decode_repl_vec<false, false, 8, true>;
+    }
+    if (ef) return (const void *)k_decode_scalar<true, true, true>;
+    return store ? (const void *)k_decode_scalar<false, true, true> : (const void *)k_decode_scalar<false, false, true>;
+}
+
+// a bfloat16 row allows 8-element vectors when it is 16-byte aligned with a stride multiple of 8
+inline int vec_width_bf16(const void *p, int64_t stride, uint32_t P)
+{
+    return (aligned(p, 16) && (P == 1 || stride % 8 == 0)) ? 8 : 0;
+}
+
 template <int VW, bool REPL>
 const void *select_dense_p(uint32_t P)
 {
@@ -538,6 +577,46 @@ extern "C" int a2sgd_step(a2sgd_ctx *c, float *w, int64_t w_stride, const float 
                                  c->global_means, s);
     if (r1) return r1;
     return launch_decode(c, w, ws, grad, grad_stride, err, err_stride, c->local_means, c->global_means, lr, s);
+}
+
+extern "C" int a2sgd_step_bf16(a2sgd_ctx *c, float *w, int64_t w_stride, const uint16_t *grad, int64_t grad_stride,
+                               float *err, int64_t err_stride, float lr, void *stream)
+{
+    if (!c || !w || !grad) return A2SGD_ERR_ARG;
+    if (!c->alg1 && !err) return A2SGD_ERR_ARG;
+    if (!stride_ok(grad_stride, c->n, c->P) || (err && !stride_ok(err_stride, c->n, c->P))) return A2SGD_ERR_ARG;
+    if (w_stride != 0 && !stride_ok(w_stride, c->n, c->P)) return A2SGD_ERR_ARG;
+    if (!aligned(grad, 2) || (err && !aligned(err, 4)) || !aligned(w, 4)) return A2SGD_ERR_ALIGN;
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return A2SGD_ERR_CUDA;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const bool ef = !c->alg1;
+    const bool store = ef || err != nullptr;
+    const int64_t ws = (c->P == 1) ? 0 : w_stride;
+    const float *g = reinterpret_cast<const float *>(grad); // element type is carried by the kernel template
+    int vw_enc = vec_width_bf16(grad, grad_stride, c->P);
+    if (ef && vec_width(err, err_stride, c->P) < 8) vw_enc = 0;
+    int vw_dec = vw_enc;
+    if (vec_width(err, err_stride, c->P) < 8 || vec_width(w, ws == 0 ? 8 : ws, c->P) < 8) vw_dec = 0;
+    {
+        EncodeArgs a = make_encode_args(c, g, grad_stride, err, err_stride, c->local_means, c->pos_counts, nullptr,
+                                        c->global_means);
+        const void *fn = select_encode_bf16(ef, vw_enc);
+        const uint64_t items = vw_enc ? (c->n + 7) / 8 : c->n;
+        const dim3 grid(std::min(per_worker_grid(c, occupancy(c, fn), items, A2SGD_WAVES_K1), c->g_alloc), c->P);
+        void *params[] = {&a};
+        A2_CUDA(launch_pdl(fn, grid, params, s));
+    }
+    {
+        DecodeArgs a = make_decode_args(c, w, ws, g, grad_stride, err, err_stride, c->local_means, c->global_means, lr);
+        const void *fn = select_decode_bf16(ef, store, ws == 0, c->P, vw_dec);
+        const uint64_t items = vw_dec ? (c->n + 7) / 8 : c->n;
+        const dim3 grid = (ws == 0) ? dim3(flat_grid(c, occupancy(c, fn), items, A2SGD_WAVES_K3))
+                                    : dim3(per_worker_grid(c, occupancy(c, fn), items, A2SGD_WAVES_K3), c->P);
+        void *params[] = {&a};
+        A2_CUDA(launch_pdl(fn, grid, params, s));
+    }
+    return A2SGD_OK;
 }
 
 extern "C" int a2sgd_dense_sync(a2sgd_ctx *c, float *w, int64_t w_stride, const float *grad, int64_t grad_stride,

@@ -122,6 +122,46 @@ __device__ __forceinline__ void st_stream1(float *p, float v)
     asm volatile("st.global.L1::no_allocate.f32 [%0], %1;" ::"l"(p), "f"(v) : "memory");
 }
 
+// A gradient row whose elements are fp32 (GB = false) or bfloat16 (GB = true; the paper notes that
+// the method "can be further integrated with quantization").  bfloat16 is the upper half of an
+// fp32, so widening is exact: v = float(g) + e is formed from exactly the value the caller stored.
+template <bool GB>
+struct GradRow {
+    const char *base;
+    __device__ __forceinline__ GradRow(const float *grad_base, int64_t row_offset_elems)
+        : base(reinterpret_cast<const char *>(grad_base) + row_offset_elems * (GB ? 2 : 4))
+    {
+    }
+    __device__ __forceinline__ float one(uint64_t elem) const
+    {
+        if (GB) {
+            unsigned short h;
+            asm volatile("ld.global.L1::no_allocate.u16 %0, [%1];" : "=h"(h) : "l"(base + 2 * elem));
+            return __uint_as_float((unsigned)h << 16);
+        }
+        return ld_stream1(reinterpret_cast<const float *>(base) + elem);
+    }
+    template <int VW>
+    __device__ __forceinline__ Vec<VW> vec(uint64_t elem) const
+    {
+        if (GB) {
+            static_assert(!GB || VW == 8, "bfloat16 gradients use 8-element (128-bit) vectors");
+            unsigned x[4];
+            asm volatile("ld.global.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                         : "=r"(x[0]), "=r"(x[1]), "=r"(x[2]), "=r"(x[3])
+                         : "l"(base + 2 * elem));
+            Vec<VW> r;
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                r.v[2 * k] = __uint_as_float(x[k] << 16);
+                r.v[2 * k + 1] = __uint_as_float(x[k] & 0xffff0000u);
+            }
+            return r;
+        }
+        return ld_vec<VW>(reinterpret_cast<const float *>(base) + elem);
+    }
+};
+
 // ------------------------------------------------------------------ per-element arithmetic
 // The partition of Section 3.1: positive group is the IEEE comparison v >= 0
 // (+0 and -0 are positive, NaN is not).  Flush-to-zero must stay off: a
@@ -300,7 +340,7 @@ __device__ __forceinline__ void finish_worker(const EncodeArgs &a, uint32_t p, d
 // 32/VW (= one 32-element mask word) whose loop bounds are uniform across the
 // group, so the sub-warp shuffles that assemble a mask word always see the
 // whole group.
-template <bool EF, bool MASK, int VW>
+template <bool EF, bool MASK, int VW, bool GB = false>
 __global__ void __launch_bounds__(kBlock) k_encode_vec(EncodeArgs a)
 {
     pdl_wait_prior_grid();
@@ -313,7 +353,7 @@ __global__ void __launch_bounds__(kBlock) k_encode_vec(EncodeArgs a)
     __shared__ int sh_flag;
 
     const uint32_t p = blockIdx.y;
-    const float *__restrict__ g = a.grad + (int64_t)p * a.grad_stride;
+    const GradRow<GB> g(a.grad, (int64_t)p * a.grad_stride);
     const float *__restrict__ e = EF ? a.err + (int64_t)p * a.err_stride : nullptr;
     const uint64_t nv = a.n / VW;
     const uint64_t full_words = a.n >> 5;
@@ -341,7 +381,7 @@ __global__ void __launch_bounds__(kBlock) k_encode_vec(EncodeArgs a)
     for (; (j - sub + (LPW - 1)) + (U - 1) * stride < nv; j += U * stride) {
         Vec<VW> gv[U], ev[U];
 #pragma unroll
-        for (int u = 0; u < U; ++u) gv[u] = ld_vec<VW>(g + VW * (j + u * stride));
+        for (int u = 0; u < U; ++u) gv[u] = g.template vec<VW>(VW * (j + u * stride));
         if (EF) {
 #pragma unroll
             for (int u = 0; u < U; ++u) ev[u] = ld_vec<VW>(e + VW * (j + u * stride));
@@ -363,7 +403,7 @@ __global__ void __launch_bounds__(kBlock) k_encode_vec(EncodeArgs a)
         float sp = 0.f, sn = 0.f;
         unsigned bits = 0;
         if (j < nv) {
-            Vec<VW> v = ld_vec<VW>(g + VW * j);
+            Vec<VW> v = g.template vec<VW>(VW * j);
             if (EF) v = add_vec<VW>(v, ld_vec<VW>(e + VW * j));
             split_vec<VW>(v, sp, sn, acc.n_pos, bits);
         }
@@ -375,7 +415,7 @@ __global__ void __launch_bounds__(kBlock) k_encode_vec(EncodeArgs a)
         // the n % VW trailing elements
         const uint64_t i = nv * VW + threadIdx.x;
         if (threadIdx.x < VW && i < a.n) {
-            float v = ld_stream1(g + i);
+            float v = g.one(i);
             if (EF) v += ld_stream1(e + i);
             float sp, sn;
             unsigned bit;
@@ -388,7 +428,7 @@ __global__ void __launch_bounds__(kBlock) k_encode_vec(EncodeArgs a)
             const uint64_t i2 = (full_words << 5) + lane;
             bool pos = false;
             if (i2 < a.n) {
-                float v = ld_stream1(g + i2);
+                float v = g.one(i2);
                 if (EF) v += ld_stream1(e + i2);
                 pos = v >= 0.0f;
             }
@@ -403,7 +443,7 @@ __global__ void __launch_bounds__(kBlock) k_encode_vec(EncodeArgs a)
 }
 
 // General path: any 4-byte alignment, scalar coalesced accesses.  grid = (G, P).
-template <bool EF, bool MASK>
+template <bool EF, bool MASK, bool GB = false>
 __global__ void __launch_bounds__(kBlock) k_encode_scalar(EncodeArgs a)
 {
     pdl_wait_prior_grid();
@@ -414,7 +454,7 @@ __global__ void __launch_bounds__(kBlock) k_encode_scalar(EncodeArgs a)
     __shared__ int sh_flag;
 
     const uint32_t p = blockIdx.y;
-    const float *__restrict__ g = a.grad + (int64_t)p * a.grad_stride;
+    const GradRow<GB> g(a.grad, (int64_t)p * a.grad_stride);
     const float *__restrict__ e = EF ? a.err + (int64_t)p * a.err_stride : nullptr;
     uint32_t *mask = MASK ? a.pos_mask + (uint64_t)p * ((a.n + 31) >> 5) : nullptr;
     const unsigned lane = threadIdx.x & 31u;
@@ -424,7 +464,7 @@ __global__ void __launch_bounds__(kBlock) k_encode_scalar(EncodeArgs a)
         float sp = 0.f, sn = 0.f;
         unsigned bit = 0;
         if (i < a.n) {
-            float v = ld_stream1(g + i);
+            float v = g.one(i);
             if (EF) v += ld_stream1(e + i);
             split1(v, sp, sn, acc.n_pos, bit);
         }
@@ -549,7 +589,7 @@ __device__ __forceinline__ Vec<VW> zero_vec()
 // workers in order (fixed summation order), so w is read and written once
 // per model element.  PT > 0: P known at compile time (all 2P+1 loads of a
 // vector are issued before any is used); PT == 0: run-time P.
-template <bool EF, bool STORE, int PT, int VW>
+template <bool EF, bool STORE, int PT, int VW, bool GB = false>
 __global__ void __launch_bounds__(kBlock) k_decode_shared_vec(DecodeArgs a)
 {
     pdl_wait_prior_grid();
@@ -578,7 +618,7 @@ __global__ void __launch_bounds__(kBlock) k_decode_shared_vec(DecodeArgs a)
                 Vec<VW> gv[PB], ev[PB];
 #pragma unroll
                 for (int q = 0; q < PB; ++q)
-                    gv[q] = ld_vec<VW>(a.grad + (int64_t)(p0 + q) * a.grad_stride + VW * j);
+                    gv[q] = GradRow<GB>(a.grad, (int64_t)(p0 + q) * a.grad_stride).template vec<VW>(VW * j);
                 if (EF) {
 #pragma unroll
                     for (int q = 0; q < PB; ++q)
@@ -602,7 +642,7 @@ __global__ void __launch_bounds__(kBlock) k_decode_shared_vec(DecodeArgs a)
             const Vec<VW> wv = ld_vec<VW>(a.w + VW * j);
             Vec<VW> sum = zero_vec<VW>();
             for (uint32_t p = 0; p < P; ++p) {
-                Vec<VW> v = ld_vec<VW>(a.grad + (int64_t)p * a.grad_stride + VW * j);
+                Vec<VW> v = GradRow<GB>(a.grad, (int64_t)p * a.grad_stride).template vec<VW>(VW * j);
                 if (EF) v = add_vec<VW>(v, ld_vec<VW>(a.err + (int64_t)p * a.err_stride + VW * j));
                 Vec<VW> gh, rs;
                 decode_vec<EF, VW>(v, sh_c[p], gh, rs);
@@ -619,7 +659,7 @@ __global__ void __launch_bounds__(kBlock) k_decode_shared_vec(DecodeArgs a)
             float sum = 0.f;
             for (uint32_t p = 0; p < P; ++p) {
                 const WorkerConst c = worker_const<EF>(a, p, m_pos, m_neg);
-                float v = ld_stream1(a.grad + (int64_t)p * a.grad_stride + i);
+                float v = GradRow<GB>(a.grad, (int64_t)p * a.grad_stride).one(i);
                 if (EF) v += ld_stream1(a.err + (int64_t)p * a.err_stride + i);
                 float gh, rs;
                 decode1<EF>(v, c, gh, rs);
@@ -632,7 +672,7 @@ __global__ void __launch_bounds__(kBlock) k_decode_shared_vec(DecodeArgs a)
 }
 
 // One w replica per worker (Algorithm 1's layout).  grid = (G, P).
-template <bool EF, bool STORE, int VW>
+template <bool EF, bool STORE, int VW, bool GB = false>
 __global__ void __launch_bounds__(kBlock) k_decode_repl_vec(DecodeArgs a)
 {
     pdl_wait_prior_grid();
@@ -641,7 +681,7 @@ __global__ void __launch_bounds__(kBlock) k_decode_repl_vec(DecodeArgs a)
     const uint32_t p = blockIdx.y;
     const float m_pos = __ldg(a.global_means), m_neg = __ldg(a.global_means + 1);
     const WorkerConst c = worker_const<EF>(a, p, m_pos, m_neg);
-    const float *__restrict__ g = a.grad + (int64_t)p * a.grad_stride;
+    const GradRow<GB> g(a.grad, (int64_t)p * a.grad_stride);
     float *e = (EF || STORE) ? a.err + (int64_t)p * a.err_stride : nullptr;
     float *w = a.w + (int64_t)p * a.w_stride;
     const float neg_lr = -a.lr;
@@ -652,7 +692,7 @@ __global__ void __launch_bounds__(kBlock) k_decode_repl_vec(DecodeArgs a)
     for (; j + (U - 1) * stride < nv; j += U * stride) {
         Vec<VW> gv[U], ev[U], wv[U];
 #pragma unroll
-        for (int u = 0; u < U; ++u) gv[u] = ld_vec<VW>(g + VW * (j + u * stride));
+        for (int u = 0; u < U; ++u) gv[u] = g.template vec<VW>(VW * (j + u * stride));
         if (EF) {
 #pragma unroll
             for (int u = 0; u < U; ++u) ev[u] = ld_vec<VW>(e + VW * (j + u * stride));
@@ -669,7 +709,7 @@ __global__ void __launch_bounds__(kBlock) k_decode_repl_vec(DecodeArgs a)
         }
     }
     for (; j < nv; j += stride) {
-        Vec<VW> v = ld_vec<VW>(g + VW * j);
+        Vec<VW> v = g.template vec<VW>(VW * j);
         if (EF) v = add_vec<VW>(v, ld_vec<VW>(e + VW * j));
         const Vec<VW> wv = ld_vec<VW>(w + VW * j);
         Vec<VW> gh, rs;
@@ -680,7 +720,7 @@ __global__ void __launch_bounds__(kBlock) k_decode_repl_vec(DecodeArgs a)
     if (blockIdx.x == 0 && threadIdx.x < VW) {
         const uint64_t i = nv * VW + threadIdx.x;
         if (i < a.n) {
-            float v = ld_stream1(g + i);
+            float v = g.one(i);
             if (EF) v += ld_stream1(e + i);
             float gh, rs;
             decode1<EF>(v, c, gh, rs);
@@ -692,7 +732,7 @@ __global__ void __launch_bounds__(kBlock) k_decode_repl_vec(DecodeArgs a)
 
 // General path: any 4-byte alignment, both weight layouts, scalar accesses.
 // Shared w: grid = (G, 1), the thread walks the workers; replicas: grid = (G, P).
-template <bool EF, bool STORE>
+template <bool EF, bool STORE, bool GB = false>
 __global__ void __launch_bounds__(kBlock) k_decode_scalar(DecodeArgs a)
 {
     pdl_wait_prior_grid();
@@ -707,7 +747,7 @@ __global__ void __launch_bounds__(kBlock) k_decode_scalar(DecodeArgs a)
         float sum = 0.f;
         for (uint32_t p = p_lo; p < p_hi; ++p) {
             const WorkerConst c = worker_const<EF>(a, p, m_pos, m_neg);
-            float v = ld_stream1(a.grad + (int64_t)p * a.grad_stride + i);
+            float v = GradRow<GB>(a.grad, (int64_t)p * a.grad_stride).one(i);
             if (EF) v += ld_stream1(a.err + (int64_t)p * a.err_stride + i);
             float gh, rs;
             decode1<EF>(v, c, gh, rs);

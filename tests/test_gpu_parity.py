@@ -479,3 +479,56 @@ def test_compressed_iterations_then_dense_sync_like_algorithm_1():
     from parity_util import count_outliers, tau_w
     assert count_outliers(w.cpu().numpy(), w_ref, tau_w(w_ref)) == 0
     ctx.destroy()
+
+
+def _widen_bf16(t):
+    """bfloat16 -> fp32 by the definition of the format (upper 16 bits of an fp32), in numpy."""
+    u16 = t.view(torch.int16).cpu().numpy().view(np.uint16)
+    return (u16.astype(np.uint32) << 16).view(np.float32)
+
+
+@pytest.mark.parametrize("mode", [EF, ALG1])
+@pytest.mark.parametrize("replicated", [False, True])
+@pytest.mark.parametrize("P,n,stride_pad,off", [(1, 9, 0, 0), (4, 1 << 20, 0, 0), (4, 100_003, 5, 0), (3, 70_000, 0, 0),
+                                                (8, 33_333, 3, 1), (2, 4096, 0, 3), (16, 2051, 13, 0)])
+def test_bf16_gradient_step_matches_oracle_on_widened_gradients(mode, replicated, P, n, stride_pad, off):
+    gen = torch.Generator("cuda").manual_seed(n + P)
+    stride = n + stride_pad
+    gbuf = torch.zeros(off + P * stride + 8, device="cuda")
+    gbuf.normal_(0.0, 1e-3, generator=gen)
+    g16_all = gbuf.to(torch.bfloat16)
+    g16 = g16_all[off:off + P * stride].view(P, stride)[:, :n]
+    assert np.array_equal(_widen_bf16(g16.contiguous()), g16.float().cpu().numpy())   # widening is exact
+    e = torch.empty((P, stride), device="cuda")[:, :n]
+    e.normal_(0.0, 3e-4, generator=gen)
+    w = (torch.empty((P, stride), device="cuda")[:, :n] if replicated else torch.empty(n, device="cuda"))
+    w.normal_(0.0, 0.02, generator=gen)
+    gh = _widen_bf16(g16.contiguous()).reshape(P, n)
+    eh, wh = e.cpu().numpy().copy(), w.cpu().numpy().copy()
+    ctx = B.a2sgd_create(n, P, 0, mode)
+    B.a2sgd_step_bf16(ctx, w, g16, e, 0.1)
+    lm, gm, cnt, status = B.a2sgd_read_stats(ctx)
+    lm_ref, gm_ref, cnt_ref = oracle.step(wh, gh, eh, 0.1, mode=mode)
+    assert status == B.OK and np.array_equal(cnt, cnt_ref)
+    assert_means(lm, lm_ref)
+    assert_means(gm, gm_ref)
+    assert_state(w.cpu().numpy(), wh, e.cpu().numpy(), eh, gm_ref, f"bf16 P={P} n={n}")
+    assert torch.equal(g16_all, gbuf.to(torch.bfloat16))      # gradients untouched
+    ctx.destroy()
+
+
+def test_maximum_worker_count():
+    """P = 1024 (the documented maximum): run-time-P kernels, one or two CTAs per worker in K1."""
+    P, n = 1024, 3001
+    views, raw, stride = _state(31, P, n, pad=3)
+    g, e, w = _host(views)
+    ctx = B.a2sgd_create(n, P, 0, EF)
+    B.a2sgd_step(ctx, views["w"], views["g"], views["e"], 0.1)
+    lm, gm, cnt, status = B.a2sgd_read_stats(ctx)
+    lm_ref, gm_ref, cnt_ref = oracle.step(w, g, e, 0.1, mode=EF)
+    assert status == B.OK and np.array_equal(cnt, cnt_ref)
+    assert_means(lm, lm_ref)
+    assert_means(gm, gm_ref)
+    assert_state(views["w"].cpu().numpy(), w, views["e"].cpu().numpy(), e, gm_ref, "P=1024")
+    _guards_intact(raw, views, n, stride, {"g": P, "e": P, "w": 1})
+    ctx.destroy()
