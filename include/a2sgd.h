@@ -72,7 +72,10 @@ enum a2sgd_flags {
     A2SGD_MODE_EF = 0,                /* default */
     A2SGD_MODE_ALG1 = 1,
     A2SGD_FORCE_TWO_PASS = 1 << 4,    /* a2sgd_step never takes the single-launch path */
-    A2SGD_FORCE_COOPERATIVE = 1 << 5, /* a2sgd_step always takes it; A2SGD_ERR_TOO_LARGE if it cannot */
+    A2SGD_FORCE_COOPERATIVE = 1 << 5, /* a2sgd_step takes the single-launch path whenever (n, P) fits it — v in
+                                         registers, or g, e, w within 70 % of L2 — and returns
+                                         A2SGD_ERR_TOO_LARGE otherwise.  Without this flag the single launch is
+                                         used only where it measured faster: one worker, v in registers. */
     A2SGD_TEST_BARRIER_NEVER_OPENS = 1 << 9 /* test hook: the single-launch path waits for one arrival more
                                                than its grid has, with a ~0.2 ms limit, so every CTA gives up,
                                                writes nothing and A2SGD_ERR_TIMEOUT is latched */
@@ -118,9 +121,9 @@ int a2sgd_decode_update(a2sgd_ctx *ctx, float *w, int64_t w_stride,
 
 /* One whole loop body of Algorithm 1 (lines 3-7) for all P workers: encode,
  * average the 2P scalars, decode/update.  The means stay in the context and
- * can be read back with a2sgd_read_stats.  Two launches for large n; a
- * single cooperative launch that keeps v on chip when n*P is small enough
- * (see a2sgd_flags). */
+ * can be read back with a2sgd_read_stats.  Two launches in general; a single
+ * cooperative launch (v kept in registers between the two phases, or, with
+ * A2SGD_FORCE_COOPERATIVE, re-read from L2) for small n*P, see a2sgd_flags. */
 int a2sgd_step(a2sgd_ctx *ctx, float *w, int64_t w_stride,
                const float *grad, int64_t grad_stride,
                float *err, int64_t err_stride, float lr, void *stream);

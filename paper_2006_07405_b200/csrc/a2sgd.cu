@@ -40,6 +40,7 @@ struct a2sgd_ctx {
     bool alg1 = false;
     int sm_count = 0;
     bool coop_supported = false;
+    size_t l2_bytes = 0;
     // scratch (device)
     Partial *partials = nullptr;
     uint32_t g_alloc = 0; // CTAs per worker the partials array can hold
@@ -280,6 +281,25 @@ const void *select_coop_p(uint32_t P)
     }
 }
 
+template <bool EF, bool STORE, bool SHARED>
+const void *select_coop_l2_p(uint32_t P)
+{
+    switch (P) {
+    case 1: return (const void *)k_step_coop_l2<EF, STORE, 1, SHARED>;
+    case 2: return (const void *)k_step_coop_l2<EF, STORE, 2, SHARED>;
+    case 4: return (const void *)k_step_coop_l2<EF, STORE, 4, SHARED>;
+    case 8: return (const void *)k_step_coop_l2<EF, STORE, 8, SHARED>;
+    default: return nullptr;
+    }
+}
+
+const void *select_coop_l2(bool ef, bool store, bool shared, uint32_t P)
+{
+    if (ef) return shared ? select_coop_l2_p<true, true, true>(P) : select_coop_l2_p<true, true, false>(P);
+    if (store) return shared ? select_coop_l2_p<false, true, true>(P) : select_coop_l2_p<false, true, false>(P);
+    return shared ? select_coop_l2_p<false, false, true>(P) : select_coop_l2_p<false, false, false>(P);
+}
+
 const void *select_coop(bool ef, bool store, bool shared, uint32_t P)
 {
     if (ef) return shared ? select_coop_p<true, true, true>(P) : select_coop_p<true, true, false>(P);
@@ -384,22 +404,44 @@ int launch_decode(a2sgd_ctx *c, float *w, int64_t ws, const float *grad, int64_t
     return A2SGD_OK;
 }
 
-// The single-launch path holds at most kCoopVecPerThread 128-bit vectors of v per thread.
+// The single-launch path.  Register-resident form: at most kCoopVecPerThread 128-bit vectors of v
+// per thread.  L2-resident form: g, e and w together within 70 % of the L2 capacity.
 // Returns the kernel and its grid, or nullptr when (n, P, alignment) does not qualify.
+//
+// Which sizes take it by default is decided by measurement (B200, CUDA graphs of 20 steps, us per
+// step, single launch vs two launches): P = 1: 1 M 9.6 vs 10.6, 2 M 11.2 vs 14.5 (register form);
+// 4 M 18.4 vs 18.1 (L2 form).  P = 2, 0.5 M: 11.1 vs 10.1.  P = 4: 0.25 M 11.0 vs 10.6, 0.5 M 13.6
+// vs 12.5, 1 M (L2 form) 17.1 vs 15.8.  The two-launch path hands its decode work to the hardware
+// CTA scheduler one vector per thread, which balances the SMs better than the equal static shares
+// a co-resident grid must use, and that outweighs the saved launch except for a single worker with
+// v in registers.  So: automatic only for P = 1 in the register form; everything else that fits is
+// available through A2SGD_FORCE_COOPERATIVE.
 const void *coop_plan(a2sgd_ctx *c, bool store, bool shared, int vw, uint32_t *grid_out)
 {
     if (!c->coop_supported || vw < 4) return nullptr;
+    const bool forced = (c->flags & A2SGD_FORCE_COOPERATIVE) != 0;
+    if (!forced && c->P != 1) return nullptr;
     const void *fn = select_coop(!c->alg1, store, shared, c->P);
     if (!fn) return nullptr;
-    const uint64_t threads = (uint64_t)c->sm_count * occupancy(c, fn) * kBlock;
-    const uint64_t per_thread = kCoopVecPerThread / c->P;
     const uint64_t n4 = (c->n + 3) / 4;
-    if (n4 > threads * per_thread) return nullptr;
     const uint64_t need = std::max<uint64_t>(1, (n4 + kBlock - 1) / kBlock);
-    const uint64_t grid = std::min<uint64_t>((uint64_t)c->sm_count * occupancy(c, fn), need);
-    if (grid > c->g_alloc) return nullptr;
+    {
+        const uint64_t resident = (uint64_t)c->sm_count * occupancy(c, fn);
+        const uint64_t per_thread = kCoopVecPerThread / c->P;
+        const uint64_t grid = std::min<uint64_t>(resident, need);
+        if (n4 <= resident * kBlock * per_thread && grid <= c->g_alloc) {
+            *grid_out = (uint32_t)grid;
+            return fn;
+        }
+    }
+    if (!forced) return nullptr;
+    const void *fn2 = select_coop_l2(!c->alg1, store, shared, c->P);
+    const uint64_t rows = (uint64_t)c->P * (c->alg1 ? (store ? 2 : 1) : 2) + (shared ? 1 : c->P);
+    const double footprint = (double)rows * (double)c->n * 4.0;
+    if (!fn2 || footprint > 0.70 * (double)c->l2_bytes) return nullptr;
+    const uint64_t grid = std::min<uint64_t>(std::min<uint64_t>((uint64_t)c->sm_count * occupancy(c, fn2), need), c->g_alloc);
     *grid_out = (uint32_t)grid;
-    return fn;
+    return fn2;
 }
 
 int launch_coop(a2sgd_ctx *c, const void *fn, uint32_t grid, float *w, int64_t ws, const float *grad, int64_t gs,
@@ -463,6 +505,9 @@ extern "C" int a2sgd_create(a2sgd_ctx **out, uint64_t n, uint32_t P, int device,
         int coop = 0;
         if (cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, device) != cudaSuccess) (void)cudaGetLastError();
         c->coop_supported = coop != 0;
+        int l2 = 0;
+        if (cudaDeviceGetAttribute(&l2, cudaDevAttrL2CacheSize, device) != cudaSuccess) (void)cudaGetLastError();
+        c->l2_bytes = (size_t)std::max(l2, 0);
     }
     // partials: room for a (G, P) grid that fills the device at the highest possible occupancy
     const uint32_t max_slots = (uint32_t)c->sm_count * (2048 / kBlock) * A2SGD_WAVES_K1;

@@ -866,13 +866,169 @@ __device__ __forceinline__ void st_release_u32(unsigned int *p, unsigned int v)
     asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
 
+// Shared memory of the single-launch kernels' reduction and barrier.
+template <int PT>
+struct CoopShared {
+    double part[PT][2][kWarps];
+    unsigned long long cnt[PT][kWarps];
+    float mu[PT][2];
+    int flag;
+};
+
+__device__ __forceinline__ void warp_reduce3(double &s_pos, double &s_neg, unsigned long long &n_pos, int width)
+{
+    for (int off = width / 2; off > 0; off >>= 1) {
+        s_pos += shfl_down_f64(s_pos, off);
+        s_neg += shfl_down_f64(s_neg, off);
+        n_pos += __shfl_down_sync(0xffffffffu, n_pos, off);
+    }
+}
+
+// Block reduction of all PT workers at once (warp w finishes worker w), partial sums to scratch,
+// grid barrier.  The last CTA to arrive folds the partials — all workers at the same time, each by
+// its own group of warps in a fixed order — publishes the local and global means and opens the
+// barrier; the others poll a release word a bounded number of times.  Returns false in a CTA that
+// gave up.  PT <= kWarps.
+template <int PT>
+__device__ __forceinline__ bool coop_reduce_and_barrier(const CoopArgs &a, Acc (&acc)[PT], CoopShared<PT> &sh)
+{
+    static_assert(PT <= kWarps, "one warp per worker");
+    const EncodeArgs &ea = a.enc;
+    const uint32_t G = gridDim.x;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#pragma unroll
+    for (int p = 0; p < PT; ++p) {
+        double s_pos = acc[p].s_pos, s_neg = acc[p].s_neg;
+        unsigned long long n_pos = acc[p].n_pos;
+        warp_reduce3(s_pos, s_neg, n_pos, 32);
+        if (lane == 0) {
+            sh.part[p][0][warp] = s_pos;
+            sh.part[p][1][warp] = s_neg;
+            sh.cnt[p][warp] = n_pos;
+        }
+    }
+    __syncthreads();
+    if (warp < PT) {
+        double s_pos = lane < kWarps ? sh.part[warp][0][lane] : 0.0;
+        double s_neg = lane < kWarps ? sh.part[warp][1][lane] : 0.0;
+        unsigned long long n_pos = lane < kWarps ? sh.cnt[warp][lane] : 0ull;
+        warp_reduce3(s_pos, s_neg, n_pos, kWarps);
+        if (lane == 0) {
+            Partial *mine = ea.partials + (uint64_t)warp * G;
+            mine[blockIdx.x].s_pos = s_pos;
+            mine[blockIdx.x].s_neg = s_neg;
+            mine[blockIdx.x].n_pos = n_pos;
+        }
+    }
+    __syncthreads();
+    // ---- grid barrier (one fence per CTA: fences are the expensive part of this path)
+    if (threadIdx.x == 0) {
+        __threadfence();
+        const unsigned int t = atomicAdd(&a.barrier[0], 1u);
+        sh.flag = (t == a.expected - 1) ? 1 : 0;
+    }
+    __syncthreads();
+    if (sh.flag) {
+        __threadfence();
+        // kWarps / PT warps fold each worker's G partials: thread tg of the group takes partials
+        // tg, tg + group size, ... (index order), then a fixed tree inside the group
+        constexpr int WPW = kWarps / PT;
+        const int worker = warp / WPW, warp_in_group = warp % WPW;
+        if (worker < PT) {
+            const Partial *part = ea.partials + (uint64_t)worker * G;
+            double fp = 0.0, fn = 0.0;
+            unsigned long long fc = 0;
+#pragma unroll 4
+            for (uint32_t i = warp_in_group * 32 + lane; i < G; i += WPW * 32) {
+                fp += __ldcg(&part[i].s_pos);
+                fn += __ldcg(&part[i].s_neg);
+                fc += __ldcg(&part[i].n_pos);
+            }
+            warp_reduce3(fp, fn, fc, 32);
+            if (lane == 0) {
+                sh.part[worker][0][warp_in_group] = fp;
+                sh.part[worker][1][warp_in_group] = fn;
+                sh.cnt[worker][warp_in_group] = fc;
+            }
+        }
+        __syncthreads();
+        if (warp < PT) {
+            double fp = lane < WPW ? sh.part[warp][0][lane] : 0.0;
+            double fn = lane < WPW ? sh.part[warp][1][lane] : 0.0;
+            unsigned long long fc = lane < WPW ? sh.cnt[warp][lane] : 0ull;
+            warp_reduce3(fp, fn, fc, kWarps);
+            if (lane == 0) {
+                const unsigned long long n_neg = ea.n - fc;
+                const float mu_pos = fc ? (float)(fp / (double)fc) : 0.0f;
+                const float mu_neg = n_neg ? (float)(fn / (double)n_neg) : 0.0f;
+                sh.mu[warp][0] = mu_pos;
+                sh.mu[warp][1] = mu_neg;
+                ea.local_means[2 * warp + 0] = mu_pos;
+                ea.local_means[2 * warp + 1] = mu_neg;
+                if (ea.pos_counts) ea.pos_counts[warp] = fc;
+                if (!isfinite(fp) || !isfinite(fn)) atomicCAS(ea.status, kDevOk, kDevNonFinite);
+            }
+        }
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            double gp = 0.0, gn = 0.0;
+            for (uint32_t q = 0; q < PT; ++q) { // worker order
+                gp += (double)sh.mu[q][0];
+                gn += (double)sh.mu[q][1];
+            }
+            ea.global_means[0] = (float)(gp / (double)PT);
+            ea.global_means[1] = (float)(gn / (double)PT);
+            a.barrier[0] = 0;
+            __threadfence();
+            st_release_u32(&a.barrier[1], a.epoch);
+        }
+        __syncthreads();
+    } else {
+        if (threadIdx.x == 0) {
+            unsigned int polls = 0;
+            int ok = 1;
+            while (ld_acquire_u32(&a.barrier[1]) != a.epoch) {
+                if (++polls > a.spin_limit) {
+                    ok = 0;
+                    break;
+                }
+                __nanosleep(40);
+            }
+            if (!ok) atomicCAS(ea.status, kDevOk, kDevTimeout);
+            sh.flag = ok ? 2 : -1;
+        }
+        __syncthreads();
+        if (sh.flag < 0) return false; // gave up: no output is written by this CTA
+    }
+    return true;
+}
+
+// Constants of the reconstruction for every worker, read after the barrier.
+template <bool EF, int PT>
+__device__ __forceinline__ void coop_worker_consts(const EncodeArgs &ea, WorkerConst (&c)[PT])
+{
+    const float m_pos = __ldcg(ea.global_means), m_neg = __ldcg(ea.global_means + 1);
+#pragma unroll
+    for (int p = 0; p < PT; ++p) {
+        if (EF) {
+            c[p].a_pos = m_pos;
+            c[p].a_neg = -m_neg;
+            c[p].b_pos = c[p].b_neg = 0.f;
+        } else {
+            const float mu_pos = __ldcg(ea.local_means + 2 * p), mu_neg = __ldcg(ea.local_means + 2 * p + 1);
+            c[p].a_pos = m_pos - mu_pos;
+            c[p].a_neg = mu_neg - m_neg;
+            c[p].b_pos = mu_pos;
+            c[p].b_neg = -mu_neg;
+        }
+    }
+}
+
 template <bool EF, bool STORE, int PT, bool SHARED>
 __global__ void __launch_bounds__(kBlock) k_step_coop(CoopArgs a)
 {
     constexpr int K = kCoopVecPerThread / PT;
-    __shared__ double sh_d[2][kWarps];
-    __shared__ unsigned long long sh_n[kWarps];
-    __shared__ int sh_flag;
+    __shared__ CoopShared<PT> sh;
 
     const EncodeArgs &ea = a.enc;
     const DecodeArgs &da = a.dec;
@@ -924,94 +1080,10 @@ __global__ void __launch_bounds__(kBlock) k_step_coop(CoopArgs a)
             acc[p].s_neg += (double)tn;
         }
     }
-    const uint32_t G = gridDim.x;
-#pragma unroll
-    for (int p = 0; p < PT; ++p) {
-        double s_pos = acc[p].s_pos, s_neg = acc[p].s_neg;
-        unsigned long long n_pos = acc[p].n_pos;
-        block_reduce(s_pos, s_neg, n_pos, sh_d, sh_n);
-        if (threadIdx.x == 0) {
-            Partial *mine = ea.partials + (uint64_t)p * G;
-            mine[blockIdx.x].s_pos = s_pos;
-            mine[blockIdx.x].s_neg = s_neg;
-            mine[blockIdx.x].n_pos = n_pos;
-        }
-    }
-    // ---- grid barrier: the last CTA to arrive folds the partials and opens it
-    if (threadIdx.x == 0) {
-        __threadfence();
-        const unsigned int t = atomicAdd(&a.barrier[0], 1u);
-        sh_flag = (t == a.expected - 1) ? 1 : 0;
-    }
-    __syncthreads();
-    if (sh_flag) {
-        __threadfence();
-        for (uint32_t p = 0; p < PT; ++p) {
-            const Partial *part = ea.partials + (uint64_t)p * G;
-            double fp = 0.0, fn = 0.0;
-            unsigned long long fc = 0;
-            for (uint32_t i = threadIdx.x; i < G; i += kBlock) {
-                fp += __ldcg(&part[i].s_pos);
-                fn += __ldcg(&part[i].s_neg);
-                fc += __ldcg(&part[i].n_pos);
-            }
-            __syncthreads();
-            block_reduce(fp, fn, fc, sh_d, sh_n);
-            if (threadIdx.x == 0) {
-                const unsigned long long n_neg = ea.n - fc;
-                ea.local_means[2 * p + 0] = fc ? (float)(fp / (double)fc) : 0.0f;
-                ea.local_means[2 * p + 1] = n_neg ? (float)(fn / (double)n_neg) : 0.0f;
-                if (ea.pos_counts) ea.pos_counts[p] = fc;
-                if (!isfinite(fp) || !isfinite(fn)) atomicCAS(ea.status, kDevOk, kDevNonFinite);
-            }
-        }
-        if (threadIdx.x == 0) {
-            double gp = 0.0, gn = 0.0;
-            for (uint32_t q = 0; q < PT; ++q) { // worker order
-                gp += (double)ea.local_means[2 * q + 0];
-                gn += (double)ea.local_means[2 * q + 1];
-            }
-            ea.global_means[0] = (float)(gp / (double)PT);
-            ea.global_means[1] = (float)(gn / (double)PT);
-            a.barrier[0] = 0;
-            __threadfence();
-            st_release_u32(&a.barrier[1], a.epoch);
-        }
-        __syncthreads();
-    } else {
-        if (threadIdx.x == 0) {
-            unsigned int polls = 0;
-            int ok = 1;
-            while (ld_acquire_u32(&a.barrier[1]) != a.epoch) {
-                if (++polls > a.spin_limit) {
-                    ok = 0;
-                    break;
-                }
-                __nanosleep(40);
-            }
-            if (!ok) atomicCAS(ea.status, kDevOk, kDevTimeout);
-            sh_flag = ok ? 2 : -1;
-        }
-        __syncthreads();
-        if (sh_flag < 0) return; // gave up: no output is written by this CTA
-    }
+    if (!coop_reduce_and_barrier<PT>(a, acc, sh)) return;
     // ---- phase 2: decode from registers
-    const float m_pos = __ldcg(ea.global_means), m_neg = __ldcg(ea.global_means + 1);
     WorkerConst c[PT];
-#pragma unroll
-    for (int p = 0; p < PT; ++p) {
-        if (EF) {
-            c[p].a_pos = m_pos;
-            c[p].a_neg = -m_neg;
-            c[p].b_pos = c[p].b_neg = 0.f;
-        } else {
-            const float mu_pos = __ldcg(ea.local_means + 2 * p), mu_neg = __ldcg(ea.local_means + 2 * p + 1);
-            c[p].a_pos = m_pos - mu_pos;
-            c[p].a_neg = mu_neg - m_neg;
-            c[p].b_pos = mu_pos;
-            c[p].b_neg = -mu_neg;
-        }
-    }
+    coop_worker_consts<EF, PT>(ea, c);
     const float scale = SHARED ? -da.lr / (float)PT : -da.lr;
 #pragma unroll
     for (int k = 0; k < K; ++k) {
@@ -1047,6 +1119,102 @@ __global__ void __launch_bounds__(kBlock) k_step_coop(CoopArgs a)
         for (int p = 0; p < PT; ++p) {
             float gh, rs;
             decode1<EF>(v_tail[p], c[p], gh, rs);
+            if (STORE) st_stream1(da.err + (int64_t)p * da.err_stride + i_tail, rs);
+            if (SHARED) {
+                sum += gh;
+            } else {
+                float *wp = da.w + (int64_t)p * da.w_stride + i_tail;
+                *wp = fmaf(scale, gh, *wp);
+            }
+        }
+        if (SHARED) da.w[i_tail] = fmaf(scale, sum, da.w[i_tail]);
+    }
+}
+
+// L2-resident form of the single launch: for sizes whose g, e and w together fit in L2 but not in
+// registers.  Phase 1 streams g and e (they stay in L2: 128-bit loads without an eviction hint),
+// phase 2 reads them again from L2 after the barrier, so HBM still sees each byte once.
+template <bool EF, bool STORE, int PT, bool SHARED>
+__global__ void __launch_bounds__(kBlock) k_step_coop_l2(CoopArgs a)
+{
+    __shared__ CoopShared<PT> sh;
+    const EncodeArgs &ea = a.enc;
+    const DecodeArgs &da = a.dec;
+    const uint64_t n4 = ea.n >> 2;
+    const uint64_t T = (uint64_t)gridDim.x * kBlock;
+    const uint64_t tid = (uint64_t)blockIdx.x * kBlock + threadIdx.x;
+    const bool has_tail = blockIdx.x == 0 && threadIdx.x < 4 && (n4 << 2) + threadIdx.x < ea.n;
+    const uint64_t i_tail = (n4 << 2) + threadIdx.x;
+
+    Acc acc[PT];
+    for (uint64_t j = tid; j < n4; j += T) {
+        Vec<4> gv[PT], ev[PT];
+#pragma unroll
+        for (int p = 0; p < PT; ++p) gv[p] = ld_vec<4>(ea.grad + (int64_t)p * ea.grad_stride + 4 * j);
+        if (EF) {
+#pragma unroll
+            for (int p = 0; p < PT; ++p) ev[p] = ld_vec<4>(ea.err + (int64_t)p * ea.err_stride + 4 * j);
+        }
+#pragma unroll
+        for (int p = 0; p < PT; ++p) {
+            const Vec<4> v = EF ? add_vec<4>(gv[p], ev[p]) : gv[p];
+            float sp, sn;
+            unsigned bits;
+            split_vec<4>(v, sp, sn, acc[p].n_pos, bits);
+            acc[p].s_pos += (double)sp;
+            acc[p].s_neg += (double)sn;
+        }
+    }
+    if (has_tail) {
+#pragma unroll
+        for (int p = 0; p < PT; ++p) {
+            float v = ld_stream1(ea.grad + (int64_t)p * ea.grad_stride + i_tail);
+            if (EF) v += ld_stream1(ea.err + (int64_t)p * ea.err_stride + i_tail);
+            float tp, tn;
+            unsigned bit;
+            split1(v, tp, tn, acc[p].n_pos, bit);
+            acc[p].s_pos += (double)tp;
+            acc[p].s_neg += (double)tn;
+        }
+    }
+    if (!coop_reduce_and_barrier<PT>(a, acc, sh)) return;
+    WorkerConst c[PT];
+    coop_worker_consts<EF, PT>(ea, c);
+    const float scale = SHARED ? -da.lr / (float)PT : -da.lr;
+    for (uint64_t j = tid; j < n4; j += T) {
+        Vec<4> gv[PT], ev[PT], wv[SHARED ? 1 : PT];
+#pragma unroll
+        for (int p = 0; p < PT; ++p) gv[p] = ld_vec<4>(da.grad + (int64_t)p * da.grad_stride + 4 * j);
+        if (EF) {
+#pragma unroll
+            for (int p = 0; p < PT; ++p) ev[p] = ld_vec<4>(da.err + (int64_t)p * da.err_stride + 4 * j);
+        }
+        if (SHARED) {
+            wv[0] = ld_vec<4>(da.w + 4 * j);
+        } else {
+#pragma unroll
+            for (int p = 0; p < PT; ++p) wv[SHARED ? 0 : p] = ld_vec<4>(da.w + (int64_t)p * da.w_stride + 4 * j);
+        }
+        Vec<4> sum = zero_vec<4>();
+#pragma unroll
+        for (int p = 0; p < PT; ++p) {
+            const Vec<4> v = EF ? add_vec<4>(gv[p], ev[p]) : gv[p];
+            Vec<4> gh, rs;
+            decode_vec<EF, 4>(v, c[p], gh, rs);
+            if (STORE) st_vec<4>(da.err + (int64_t)p * da.err_stride + 4 * j, rs);
+            if (SHARED) sum = add_vec<4>(sum, gh);
+            else st_vec<4>(da.w + (int64_t)p * da.w_stride + 4 * j, axpy_vec<4>(scale, gh, wv[SHARED ? 0 : p]));
+        }
+        if (SHARED) st_vec<4>(da.w + 4 * j, axpy_vec<4>(scale, sum, wv[0]));
+    }
+    if (has_tail) {
+        float sum = 0.f;
+#pragma unroll
+        for (int p = 0; p < PT; ++p) {
+            float v = ld_stream1(da.grad + (int64_t)p * da.grad_stride + i_tail);
+            if (EF) v += ld_stream1(da.err + (int64_t)p * da.err_stride + i_tail);
+            float gh, rs;
+            decode1<EF>(v, c[p], gh, rs);
             if (STORE) st_stream1(da.err + (int64_t)p * da.err_stride + i_tail, rs);
             if (SHARED) {
                 sum += gh;

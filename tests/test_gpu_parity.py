@@ -360,7 +360,9 @@ def test_host_gradient_entry_point():
 
 
 @pytest.mark.parametrize("mode", [EF, ALG1])
-@pytest.mark.parametrize("P,n", [(1, 1 << 20), (1, (1 << 20) + 3), (2, 500_001), (4, 250_000), (8, 123_457), (4, 5)])
+@pytest.mark.parametrize("P,n", [(1, 1 << 20), (1, (1 << 20) + 3), (2, 500_001), (4, 250_000), (8, 123_457), (4, 5),
+                                 # beyond the register-resident capacity: the L2-resident form
+                                 (1, 5_000_003), (2, 2_500_001), (4, 1_200_000), (8, 400_002)])
 @pytest.mark.parametrize("replicated", [False, True])
 def test_single_launch_path(mode, P, n, replicated):
     """The cooperative single-launch kernel (v kept in registers between the two phases) against
