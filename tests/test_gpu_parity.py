@@ -534,3 +534,99 @@ def test_maximum_worker_count():
     assert_state(views["w"].cpu().numpy(), w, views["e"].cpu().numpy(), e, gm_ref, "P=1024")
     _guards_intact(raw, views, n, stride, {"g": P, "e": P, "w": 1})
     ctx.destroy()
+
+
+def test_randomised_shapes_strides_alignments():
+    """Seeded random sweep over n, P, mode, weight layout, row stride and pointer offsets."""
+    rng = np.random.default_rng(20060740)
+    for trial in range(40):
+        P = int(rng.choice([1, 2, 3, 4, 5, 8, 11, 16]))
+        n = int(rng.choice([rng.integers(1, 300), rng.integers(300, 70_000), rng.integers(70_000, 400_000)]))
+        mode = int(rng.choice([EF, ALG1]))
+        replicated = bool(rng.integers(0, 2))
+        pad = int(rng.choice([0, 0, (-n) % 8, (-n) % 32, rng.integers(0, 40)]))
+        off = tuple(int(x) for x in rng.choice([0, 0, 0, 1, 2, 3, 4, 8], size=3))
+        views, raw, stride = _state(5000 + trial, P, n, pad=pad, off=off, replicated=replicated,
+                                    g_scale=float(10.0 ** rng.uniform(-5, 0)), e_scale=float(10.0 ** rng.uniform(-6, -1)))
+        g, e, w = _host(views)
+        ctx = B.a2sgd_create(n, P, 0, mode)
+        lr = float(rng.choice([0.01, 0.1, 1.0]))
+        B.a2sgd_step(ctx, views["w"], views["g"], views["e"], lr)
+        lm, gm, cnt, status = B.a2sgd_read_stats(ctx)
+        lm_ref, gm_ref, cnt_ref = oracle.step(w, g, e, lr, mode=mode)
+        what = f"trial {trial}: P={P} n={n} mode={mode} repl={replicated} pad={pad} off={off}"
+        assert status == B.OK and np.array_equal(cnt, cnt_ref), what
+        assert_means(lm, lm_ref, what)
+        assert_means(gm, gm_ref, what)
+        assert_state(views["w"].cpu().numpy(), w, views["e"].cpu().numpy(), e, gm_ref, what)
+        _guards_intact(raw, views, n, stride, {"g": P, "e": P, "w": P if replicated else 1})
+        ctx.destroy()
+
+
+def test_steps_captured_in_a_cuda_graph_replay_bitwise():
+    """The two launches of a step (programmatic dependent launch included) can be captured and
+    replayed; replays give the same bits as eager launches."""
+    wl = W.scaled(W.get_workload("c2_lstm_ptb"), 16)
+    n, P = wl.n, wl.P
+    g = B.padded_rows(P, n, "cuda")
+    W.fill_gradients(wl, 0, g)
+    w0 = torch.empty(n, device="cuda")
+    W.init_weights(wl, w0)
+
+    def run(use_graph):
+        e = B.padded_rows(P, n, "cuda", fill=0.0)
+        w = w0.clone()
+        ctx = B.a2sgd_create(n, P, 0, EF)
+        B.a2sgd_step(ctx, w, g, e, wl.lr)                     # warm-up outside any capture
+        if use_graph:
+            side = torch.cuda.Stream()
+            side.wait_stream(torch.cuda.current_stream())
+            with torch.cuda.stream(side):
+                graph = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(graph, stream=side):
+                    for _ in range(2):
+                        B.a2sgd_step(ctx, w, g, e, wl.lr, stream=side)
+            torch.cuda.current_stream().wait_stream(side)
+            graph.replay()
+            graph.replay()
+        else:
+            for _ in range(4):
+                B.a2sgd_step(ctx, w, g, e, wl.lr)
+        lm, gm, cnt, status = B.a2sgd_read_stats(ctx)
+        out = (status, lm.tobytes(), gm.tobytes(), cnt.tobytes(), w.cpu().numpy().tobytes(), e.cpu().numpy().tobytes())
+        ctx.destroy()
+        return out
+
+    eager, replayed = run(False), run(True)
+    assert eager[0] == B.OK and eager == replayed
+
+
+def test_two_contexts_on_two_streams_do_not_interfere():
+    wl = W.scaled(W.get_workload("c4_vgg16"), 32)
+    n, P = wl.n, wl.P
+    streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+    states, refs = [], []
+    for k in range(2):
+        g = B.padded_rows(P, n, "cuda")
+        W.fill_gradients(wl, k, g)
+        e = B.padded_rows(P, n, "cuda", fill=0.0)
+        w = torch.empty(n, device="cuda")
+        W.init_weights(wl, w)
+        states.append((g, e, w, B.a2sgd_create(n, P, 0, EF)))
+        gh, eh, wh = g.cpu().numpy(), e.cpu().numpy().copy(), w.cpu().numpy().copy()
+        for _ in range(3):
+            oracle.step(wh, gh, eh, wl.lr, mode=EF)
+        refs.append((eh, wh))
+    torch.cuda.synchronize()
+    for it in range(3):
+        for k in range(2):
+            g, e, w, ctx = states[k]
+            with torch.cuda.stream(streams[k]):
+                B.a2sgd_step(ctx, w, g, e, wl.lr, stream=streams[k])
+    torch.cuda.synchronize()
+    for k in range(2):
+        g, e, w, ctx = states[k]
+        lm, gm, cnt, status = B.a2sgd_read_stats(ctx)
+        assert status == B.OK
+        assert_state(w.cpu().numpy(), refs[k][1], e.cpu().numpy(), refs[k][0], gm, f"stream {k}", max_outliers=2)
+        ctx.destroy()
