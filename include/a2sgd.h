@@ -29,10 +29,13 @@
  *
  * Pointers.  Unless an argument is marked HOST it is DEVICE memory on the
  * context's device, owned by the caller, at least 4-byte aligned.  The
- * library never allocates, frees or retains these buffers.  Any alignment
- * that is a multiple of 4 bytes is computed correctly; the fast kernels
- * need 16-byte aligned bases and strides that are multiples of 4 elements.
- * `grad` is never written.
+ * library never allocates, frees or retains these buffers (a segment plan
+ * retains the pointers it was given, see a2sgd_segments_create).  Any
+ * alignment that is a multiple of 4 bytes is computed correctly: rows that
+ * are 32-byte aligned with strides that are multiples of 8 elements take the
+ * 256-bit kernels, 16-byte / 4 elements the 128-bit ones, anything else the
+ * scalar kernels.  For full speed start every row on a 128-byte boundary
+ * (stride = n rounded up to 32 elements).  `grad` is never written.
  *
  * Execution.  Every call enqueues its kernels on `stream` (a cudaStream_t
  * passed as void*, NULL = default stream) and returns without waiting, except
@@ -43,8 +46,11 @@
  * Results are bitwise reproducible for a fixed (n, P, strides' alignment,
  * device, build): no floating-point atomics, fixed-order combines.
  * A context owns only small scratch (per-CTA partial sums, 2P+2 means, P
- * counts, tickets, status); use one context per stream; a context is not
- * thread-safe.  Limits: 1 <= n < 2^40, 1 <= P <= 1024.
+ * counts, tickets, barrier words, status); use one context per stream; a
+ * context is not thread-safe.  Kernels are launched with programmatic stream
+ * serialisation and wait for the preceding grid before their first memory
+ * access, so ordinary stream order is what the caller observes.
+ * Limits: 1 <= n < 2^40, 1 <= P <= 1024.
  */
 #ifndef A2SGD_H_
 #define A2SGD_H_

@@ -94,3 +94,45 @@ def test_full_size_step_matches_oracle(name):
         scale = max(v_pos_sum, 1e-30)
         assert abs(got - expect) <= 2e-5 * scale, (name, p, got, expect)
     ctx.destroy()
+
+
+@pytest.mark.parametrize("mode,replicated", [(B.MODE_ALG1, False), (B.MODE_EF, True), (B.MODE_ALG1, True)])
+def test_full_size_other_modes_and_layouts(mode, replicated):
+    """c2 at full size in the configurations the benchmark does not time: the paper-literal
+    Algorithm 1 mode and one weight replica per worker.  Same protocol: full oracle pass for the
+    means, sampled windows for w and err."""
+    wl = W.get_workload("c2_lstm_ptb")
+    n, P = wl.n, wl.P
+    dev = torch.device("cuda:0")
+    g = B.padded_rows(P, n, dev)
+    e = B.padded_rows(P, n, dev)
+    W.fill_gradients(wl, 1, g)
+    gen = torch.Generator(device=dev).manual_seed(wl.seed + 7)
+    e.normal_(0.0, 1e-4, generator=gen)
+    if replicated:
+        w = B.padded_rows(P, n, dev)
+        w.normal_(0.0, wl.w_std, generator=gen)
+    else:
+        w = torch.empty(n, device=dev)
+        W.init_weights(wl, w)
+    ctx = B.a2sgd_create(n, P, 0, mode)
+    launch = B.a2sgd_launch_info(ctx, shared_w=not replicated)
+    idx = _sample_indices(n, launch, wl.seed + 1)
+    idx_dev = torch.from_numpy(idx).to(dev)
+    g_s = g[:, idx_dev].cpu().numpy()
+    e_s = e[:, idx_dev].cpu().numpy()
+    w_s = (w[:, idx_dev] if replicated else w[idx_dev]).cpu().numpy()
+    gh = g.cpu().numpy()
+    eh = e.cpu().numpy() if mode == B.MODE_EF else None
+    lm_ref, cnt_ref, _ = oracle.encode(gh, eh, mode=mode)
+    gm_ref = oracle.global_average(lm_ref)
+    del gh, eh
+    B.a2sgd_step(ctx, w, g, e, wl.lr)
+    lm, gm, cnt, status = B.a2sgd_read_stats(ctx)
+    assert status == B.OK and np.array_equal(cnt, cnt_ref)
+    assert_means(lm, lm_ref)
+    assert_means(gm, gm_ref)
+    oracle.decode_update(w_s, g_s, e_s, lm_ref, gm_ref, wl.lr, mode=mode)
+    w_got = (w[:, idx_dev] if replicated else w[idx_dev]).cpu().numpy()
+    assert_state(w_got, w_s, e[:, idx_dev].cpu().numpy(), e_s, gm_ref, f"mode {mode} replicated {replicated}")
+    ctx.destroy()
