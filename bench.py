@@ -302,6 +302,18 @@ def time_workload(wl, steps, warmup, dev, *, with_roofline=True, with_e2e=True, 
         evs[1].record()
         torch.cuda.synchronize(dev)
         res["dense_sync_ms"] = evs[0].elapsed_time(evs[1]) / k_steps
+        if g.stride(0) % 8 == 0:
+            dctx = B.a2sgd_create(n, P, dev.index, B.MODE_EF | B.DEFERRED_RESIDUAL)
+            for _ in range(3):
+                B.a2sgd_step(dctx, w, g, e, wl.lr)
+            evs[0].record()
+            for _ in range(k_steps):
+                B.a2sgd_step(dctx, w, g, e, wl.lr)
+            evs[1].record()
+            B.a2sgd_materialize_err(dctx, e)
+            torch.cuda.synchronize(dev)
+            res["step_deferred_ms"] = evs[0].elapsed_time(evs[1]) / k_steps
+            dctx.destroy()
         g16 = torch.empty((P, g.stride(0)), dtype=torch.bfloat16, device=dev)[:, :n]
         g16.copy_(g)
         for _ in range(3):
@@ -529,6 +541,13 @@ def main():
             "ms": res["step_segments_ms"], "GBps": bts / (res["step_segments_ms"] * 1e-3) / 1e9,
             "frac_of_8TBps": bts / (res["step_segments_ms"] * 1e-3) / 1e9 / NOMINAL_HBM_GBS,
             "segments": len(wl.segments)}
+    if "step_deferred_ms" in res:
+        bts = (12 * wl.P + 8 + wl.P / 4) * wl.n
+        next_rows["step, deferred-residual representation (opt-in, bit-identical results)"] = {
+            "ms": res["step_deferred_ms"], "GBps_actual_bytes": bts / (res["step_deferred_ms"] * 1e-3) / 1e9,
+            "model_params_per_s": wl.n / (res["step_deferred_ms"] * 1e-3),
+            "bytes_per_model_element": 12 * wl.P + 8 + wl.P / 4,
+            "speedup_vs_canonical_step": res["ms_per_step"] / res["step_deferred_ms"]}
     if "step_bf16_ms" in res:
         bts = (16 * wl.P + 8) * wl.n
         next_rows["step with bfloat16 gradients"] = {

@@ -82,6 +82,17 @@ enum a2sgd_flags {
                                          registers, or g, e, w within 70 % of L2 — and returns
                                          A2SGD_ERR_TOO_LARGE otherwise.  Without this flag the single launch is
                                          used only where it measured faster: one worker, v in registers. */
+    A2SGD_DEFERRED_RESIDUAL = 1 << 7, /* EF mode only, opt-in: between steps the caller's error buffer holds the
+                                         compensated vector v of the last step instead of the residual
+                                         e = v - g_hat(v); the subtraction is done one step later, with the
+                                         means the context kept.  Same fp32 operations, so w and (after
+                                         a2sgd_materialize_err) err are bit-identical to the default, but a
+                                         step moves (12P + 8 + P/4) bytes per model element instead of
+                                         (20P + 8).  Needs 32-byte aligned rows with strides that are multiples
+                                         of 8 (A2SGD_ERR_ALIGN otherwise), the same error buffer at every
+                                         step, and only a2sgd_step / a2sgd_step_host / a2sgd_dense_sync /
+                                         a2sgd_materialize_err on this context.  The context also owns a sign
+                                         mask of P*n/8 bytes. */
     A2SGD_TEST_BARRIER_NEVER_OPENS = 1 << 9 /* test hook: the single-launch path waits for one arrival more
                                                than its grid has, with a ~0.2 ms limit, so every CTA gives up,
                                                writes nothing and A2SGD_ERR_TIMEOUT is latched */
@@ -145,6 +156,13 @@ int a2sgd_step(a2sgd_ctx *ctx, float *w, int64_t w_stride,
 int a2sgd_step_bf16(a2sgd_ctx *ctx, float *w, int64_t w_stride,
                     const uint16_t *grad, int64_t grad_stride,
                     float *err, int64_t err_stride, float lr, void *stream);
+
+/* For contexts created with A2SGD_DEFERRED_RESIDUAL: rewrites the error buffer in place from the
+ * compensated vector v it holds after a step to the true residual e = v - g_hat(v) of that step
+ * (one pass, 8 bytes per worker-element), e.g. before a checkpoint or before handing the buffer
+ * to other code.  The next a2sgd_step then treats it as a residual again.  No-op when the buffer
+ * already holds a residual (before the first step, or right after this call). */
+int a2sgd_materialize_err(a2sgd_ctx *ctx, float *err, int64_t err_stride, void *stream);
 
 /* Algorithm 1 lines 9-10: the dense synchronisation that follows the last compressed iteration
  * (Eq. 1 for one step).  The workers' gradients are averaged element-wise, summed in worker

@@ -23,6 +23,7 @@ MODE_EF = 0
 MODE_ALG1 = 1
 FORCE_TWO_PASS = 1 << 4
 FORCE_COOPERATIVE = 1 << 5
+DEFERRED_RESIDUAL = 1 << 7
 TEST_BARRIER_NEVER_OPENS = 1 << 9
 ROW_ALIGN_ELEMS = 32   # 128 bytes: rows that start on a cache-line boundary take the widest vector kernels
 
@@ -82,6 +83,8 @@ def lib() -> ctypes.CDLL:
         l.a2sgd_step_segments.argtypes = [_vp, _vp, ctypes.c_float, _vp]
         l.a2sgd_step_bf16.restype = ctypes.c_int
         l.a2sgd_step_bf16.argtypes = [_vp, _vp, _i64, _vp, _i64, _vp, _i64, ctypes.c_float, _vp]
+        l.a2sgd_materialize_err.restype = ctypes.c_int
+        l.a2sgd_materialize_err.argtypes = [_vp, _vp, _i64, _vp]
         l.a2sgd_status_string.restype = ctypes.c_char_p
         l.a2sgd_status_string.argtypes = [ctypes.c_int]
         _lib = l
@@ -231,6 +234,12 @@ def a2sgd_step_bf16(ctx: Context, w: torch.Tensor, grad: torch.Tensor, err: Opti
     ep, es = _rows(err, "err")
     _check(lib().a2sgd_step_bf16(ctx.handle, wp, ws, grad.data_ptr(), grad.stride(0), ep, es, float(lr),
                                  _stream(stream)), "a2sgd_step_bf16")
+
+
+def a2sgd_materialize_err(ctx: Context, err: torch.Tensor, stream=None) -> None:
+    """Deferred-residual contexts: turn the buffer (holding v) back into the true residual, in place."""
+    ep, es = _rows(err, "err")
+    _check(lib().a2sgd_materialize_err(ctx.handle, ep, es, _stream(stream)), "a2sgd_materialize_err")
 
 
 def a2sgd_dense_sync(ctx: Context, w: torch.Tensor, grad: torch.Tensor, lr: float, stream=None) -> None:

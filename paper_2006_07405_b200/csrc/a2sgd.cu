@@ -25,6 +25,11 @@ using namespace a2sgd;
 #ifndef A2SGD_WAVES_K1
 #define A2SGD_WAVES_K1 2
 #endif
+#ifndef A2SGD_WAVES_K1_DEFERRED
+#define A2SGD_WAVES_K1_DEFERRED 16 /* the deferred-residual encode also writes v: a read/write mix, and like the
+                                      decode kernels it gains from many CTAs per slot (c2: 626 us per step at 1,
+                                      602 at 4, 583 at 16 and 32, 599 at 64) */
+#endif
 #ifndef A2SGD_WAVES_K3
 #define A2SGD_WAVES_K3 (1 << 20) /* effectively: cover every vector with its own thread */
 #endif
@@ -51,6 +56,10 @@ struct a2sgd_ctx {
     unsigned int *barrier = nullptr; // 2 words: arrival counter, release epoch
     int *status = nullptr;
     unsigned int coop_epoch = 0;
+    // deferred-residual representation (A2SGD_DEFERRED_RESIDUAL)
+    uint32_t *sign_mask = nullptr; // [P][ceil(n/32)]
+    float *prev_means = nullptr;   // [2]
+    bool err_holds_v = false;      // the caller's error buffer currently holds v, not e
     // resident CTAs per SM of every kernel instance used so far (occupancy API, cached)
     std::unordered_map<const void *, int> occ;
 };
@@ -462,6 +471,56 @@ int launch_coop(a2sgd_ctx *c, const void *fn, uint32_t grid, float *w, int64_t w
     return A2SGD_OK;
 }
 
+template <bool REPL>
+const void *select_decode_deferred(uint32_t P)
+{
+    switch (P) {
+    case 1: return (const void *)k_decode_deferred<1, REPL>;
+    case 2: return (const void *)k_decode_deferred<2, REPL>;
+    case 4: return (const void *)k_decode_deferred<4, REPL>;
+    case 8: return (const void *)k_decode_deferred<8, REPL>;
+    default: return (const void *)k_decode_deferred<0, REPL>;
+    }
+}
+
+// One step in the deferred-residual representation (see k_encode_vec / k_decode_deferred).
+int deferred_step(a2sgd_ctx *c, float *w, int64_t ws, const float *grad, int64_t gs, float *err, int64_t es,
+                  float lr, cudaStream_t s)
+{
+    // this form has 256-bit kernels only
+    if (vec_width(grad, gs, c->P) < 8 || vec_width(err, es, c->P) < 8 || vec_width(w, ws == 0 ? 8 : ws, c->P) < 8)
+        return A2SGD_ERR_ALIGN;
+    {
+        EncodeArgs a = make_encode_args(c, grad, gs, err, es, c->local_means, c->pos_counts, c->sign_mask,
+                                        c->global_means);
+        a.prev_means = c->prev_means;
+        const void *fn = c->err_holds_v ? (const void *)k_encode_vec<true, true, 8, false, 2>
+                                        : (const void *)k_encode_vec<true, true, 8, false, 1>;
+        const dim3 grid(std::min(per_worker_grid(c, occupancy(c, fn), (c->n + 7) / 8, A2SGD_WAVES_K1_DEFERRED), c->g_alloc), c->P);
+        void *params[] = {&a};
+        A2_CUDA(launch_pdl(fn, grid, params, s));
+    }
+    {
+        DeferredDecodeArgs a{};
+        a.w = w;
+        a.w_stride = ws;
+        a.v = err;
+        a.v_stride = es;
+        a.mask = c->sign_mask;
+        a.n = c->n;
+        a.P = c->P;
+        a.global_means = c->global_means;
+        a.prev_means = c->prev_means;
+        a.lr = lr;
+        const void *fn = ws == 0 ? select_decode_deferred<false>(c->P) : select_decode_deferred<true>(c->P);
+        const dim3 grid(flat_grid(c, occupancy(c, fn), std::max<uint64_t>(1, (c->n / 32) * 4), A2SGD_WAVES_K3));
+        void *params[] = {&a};
+        A2_CUDA(launch_pdl(fn, grid, params, s));
+    }
+    c->err_holds_v = true;
+    return A2SGD_OK;
+}
+
 int check_common(const a2sgd_ctx *c, const float *grad, int64_t gs, const float *err, int64_t es,
                  bool err_required)
 {
@@ -481,7 +540,8 @@ extern "C" int a2sgd_create(a2sgd_ctx **out, uint64_t n, uint32_t P, int device,
     if (!out) return A2SGD_ERR_ARG;
     *out = nullptr;
     const uint32_t known = A2SGD_MODE_ALG1 | A2SGD_FORCE_TWO_PASS | A2SGD_FORCE_COOPERATIVE |
-                           A2SGD_TEST_BARRIER_NEVER_OPENS;
+                           A2SGD_TEST_BARRIER_NEVER_OPENS | A2SGD_DEFERRED_RESIDUAL;
+    if ((flags & A2SGD_DEFERRED_RESIDUAL) && (flags & (A2SGD_MODE_ALG1 | A2SGD_FORCE_COOPERATIVE))) return A2SGD_ERR_ARG;
     if (n == 0 || n >= (1ull << 40) || P == 0 || P > (uint32_t)kMaxP || (flags & ~known)) return A2SGD_ERR_ARG;
     if ((flags & A2SGD_FORCE_TWO_PASS) && (flags & A2SGD_FORCE_COOPERATIVE)) return A2SGD_ERR_ARG;
     int count = 0;
@@ -510,7 +570,7 @@ extern "C" int a2sgd_create(a2sgd_ctx **out, uint64_t n, uint32_t P, int device,
         c->l2_bytes = (size_t)std::max(l2, 0);
     }
     // partials: room for a (G, P) grid that fills the device at the highest possible occupancy
-    const uint32_t max_slots = (uint32_t)c->sm_count * (2048 / kBlock) * A2SGD_WAVES_K1;
+    const uint32_t max_slots = (uint32_t)c->sm_count * (2048 / kBlock) * std::max(A2SGD_WAVES_K1, A2SGD_WAVES_K1_DEFERRED);
     c->g_alloc = std::max<uint32_t>(1, max_slots / P);
     bool ok = true;
     ok = ok && cudaMalloc(&c->partials, sizeof(Partial) * (size_t)c->g_alloc * P) == cudaSuccess;
@@ -520,6 +580,11 @@ extern "C" int a2sgd_create(a2sgd_ctx **out, uint64_t n, uint32_t P, int device,
     ok = ok && cudaMalloc(&c->tickets, sizeof(unsigned int) * (P + 1)) == cudaSuccess;
     ok = ok && cudaMalloc(&c->status, sizeof(int)) == cudaSuccess;
     ok = ok && cudaMalloc(&c->barrier, sizeof(unsigned int) * 2) == cudaSuccess;
+    if (flags & A2SGD_DEFERRED_RESIDUAL) {
+        ok = ok && cudaMalloc(&c->sign_mask, sizeof(uint32_t) * (size_t)P * ((n + 31) / 32)) == cudaSuccess;
+        ok = ok && cudaMalloc(&c->prev_means, sizeof(float) * 2) == cudaSuccess;
+        ok = ok && cudaMemset(c->prev_means, 0, sizeof(float) * 2) == cudaSuccess;
+    }
     ok = ok && cudaMemset(c->barrier, 0, sizeof(unsigned int) * 2) == cudaSuccess;
     ok = ok && cudaMemset(c->local_means, 0, sizeof(float) * 2 * P) == cudaSuccess;
     ok = ok && cudaMemset(c->global_means, 0, sizeof(float) * 2) == cudaSuccess;
@@ -547,6 +612,8 @@ extern "C" int a2sgd_destroy(a2sgd_ctx *c)
     cudaFree(c->tickets);
     cudaFree(c->status);
     cudaFree(c->barrier);
+    cudaFree(c->sign_mask);
+    cudaFree(c->prev_means);
     (void)cudaGetLastError();
     delete c;
     return A2SGD_OK;
@@ -557,6 +624,7 @@ extern "C" int a2sgd_encode(a2sgd_ctx *c, const float *grad, int64_t grad_stride
                             uint32_t *pos_mask, void *stream)
 {
     if (!c || !local_means) return A2SGD_ERR_ARG;
+    if (c->flags & A2SGD_DEFERRED_RESIDUAL) return A2SGD_ERR_ARG; // the error buffer may not hold a residual
     const int rc = check_common(c, grad, grad_stride, err, err_stride, !c->alg1);
     if (rc) return rc;
     if (!aligned(local_means, 4) || (pos_counts && !aligned(pos_counts, 8)) || (pos_mask && !aligned(pos_mask, 4)))
@@ -586,6 +654,7 @@ extern "C" int a2sgd_decode_update(a2sgd_ctx *c, float *w, int64_t w_stride, con
                                    void *stream)
 {
     if (!c || !w || !global_means) return A2SGD_ERR_ARG;
+    if (c->flags & A2SGD_DEFERRED_RESIDUAL) return A2SGD_ERR_ARG;
     const int rc = check_common(c, grad, grad_stride, err, err_stride, !c->alg1);
     if (rc) return rc;
     if (c->alg1 && !local_means) return A2SGD_ERR_ARG;
@@ -610,6 +679,7 @@ extern "C" int a2sgd_step(a2sgd_ctx *c, float *w, int64_t w_stride, const float 
     if (!guard.ok) return A2SGD_ERR_CUDA;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const int64_t ws = (c->P == 1) ? 0 : w_stride;
+    if (c->flags & A2SGD_DEFERRED_RESIDUAL) return deferred_step(c, w, ws, grad, grad_stride, err, err_stride, lr, s);
     if (!(c->flags & A2SGD_FORCE_TWO_PASS)) {
         const bool store = !c->alg1 || err != nullptr;
         const int vw = decode_vec_width(c, w, ws, grad, grad_stride, err, err_stride);
@@ -629,6 +699,7 @@ extern "C" int a2sgd_step_bf16(a2sgd_ctx *c, float *w, int64_t w_stride, const u
 {
     if (!c || !w || !grad) return A2SGD_ERR_ARG;
     if (!c->alg1 && !err) return A2SGD_ERR_ARG;
+    if (c->flags & A2SGD_DEFERRED_RESIDUAL) return A2SGD_ERR_ARG;
     if (!stride_ok(grad_stride, c->n, c->P) || (err && !stride_ok(err_stride, c->n, c->P))) return A2SGD_ERR_ARG;
     if (w_stride != 0 && !stride_ok(w_stride, c->n, c->P)) return A2SGD_ERR_ARG;
     if (!aligned(grad, 2) || (err && !aligned(err, 4)) || !aligned(w, 4)) return A2SGD_ERR_ALIGN;
@@ -661,6 +732,23 @@ extern "C" int a2sgd_step_bf16(a2sgd_ctx *c, float *w, int64_t w_stride, const u
         void *params[] = {&a};
         A2_CUDA(launch_pdl(fn, grid, params, s));
     }
+    return A2SGD_OK;
+}
+
+extern "C" int a2sgd_materialize_err(a2sgd_ctx *c, float *err, int64_t err_stride, void *stream)
+{
+    if (!c || !err) return A2SGD_ERR_ARG;
+    if (!(c->flags & A2SGD_DEFERRED_RESIDUAL)) return A2SGD_ERR_ARG;
+    if (!stride_ok(err_stride, c->n, c->P)) return A2SGD_ERR_ARG;
+    if (vec_width(err, err_stride, c->P) < 8) return A2SGD_ERR_ALIGN;
+    if (!c->err_holds_v) return A2SGD_OK; // already a true residual
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return A2SGD_ERR_CUDA;
+    const uint64_t need = std::max<uint64_t>(1, (c->n / 8 + kBlock - 1) / kBlock);
+    const dim3 grid((unsigned)std::min<uint64_t>(need, 0x7fffffffu), c->P);
+    k_materialize_err<<<grid, kBlock, 0, static_cast<cudaStream_t>(stream)>>>(err, err_stride, c->n, c->global_means);
+    A2_CUDA(cudaGetLastError());
+    c->err_holds_v = false;
     return A2SGD_OK;
 }
 
@@ -710,6 +798,7 @@ extern "C" int a2sgd_segments_create(a2sgd_ctx *c, uint32_t S, const uint64_t *n
     if (!out) return A2SGD_ERR_ARG;
     *out = nullptr;
     if (!c || S == 0 || !numel || !grad || !w) return A2SGD_ERR_ARG;
+    if (c->flags & A2SGD_DEFERRED_RESIDUAL) return A2SGD_ERR_ARG;
     if (!c->alg1 && !err) return A2SGD_ERR_ARG;
     const uint32_t P = c->P;
     const bool repl = w_replicated != 0 && P > 1;

@@ -269,6 +269,7 @@ struct EncodeArgs {
     unsigned long long *pos_counts; // [P] or nullptr
     uint32_t *pos_mask;         // [P][ceil(n/32)] or nullptr
     float *global_means;        // [2] or nullptr: fold the global average into the last CTA
+    const float *prev_means;    // [2]: last step's global means (deferred-residual form only)
     // second copies kept in the context for read_stats (may alias the above or be nullptr)
     float *ctx_local_means;
     unsigned long long *ctx_pos_counts;
@@ -340,9 +341,18 @@ __device__ __forceinline__ void finish_worker(const EncodeArgs &a, uint32_t p, d
 // 32/VW (= one 32-element mask word) whose loop bounds are uniform across the
 // group, so the sub-warp shuffles that assemble a mask word always see the
 // whole group.
-template <bool EF, bool MASK, int VW, bool GB = false>
+//
+// DEFER selects the deferred-residual representation of the error buffer (EF mode, MASK on,
+// VW = 8 only).  There the buffer holds, between steps, the compensated vector v of the last
+// step instead of the residual e' = v - g_hat(v); the residual is formed here, one step late,
+// with the previous step's global means (a.prev_means) — the same fp32 subtraction the decode
+// kernel would have done, so every value is bit-identical — and the new v is written back in
+// place.  The decode kernel then needs only the sign mask and w.  DEFER = 1: the buffer still
+// holds a true residual (first step, or after a2sgd_materialize_err); DEFER = 2: it holds v.
+template <bool EF, bool MASK, int VW, bool GB = false, int DEFER = 0>
 __global__ void __launch_bounds__(kBlock) k_encode_vec(EncodeArgs a)
 {
+    static_assert(DEFER == 0 || (EF && MASK && VW == 8 && !GB), "deferred residual: EF, mask, 256-bit, fp32 gradients");
     pdl_wait_prior_grid();
     pdl_release_next_grid();
 
@@ -354,7 +364,22 @@ __global__ void __launch_bounds__(kBlock) k_encode_vec(EncodeArgs a)
 
     const uint32_t p = blockIdx.y;
     const GradRow<GB> g(a.grad, (int64_t)p * a.grad_stride);
-    const float *__restrict__ e = EF ? a.err + (int64_t)p * a.err_stride : nullptr;
+    const float *e = EF ? a.err + (int64_t)p * a.err_stride : nullptr;
+    float *e_out = DEFER ? const_cast<float *>(e) : nullptr; // deferred form rewrites the buffer in place
+    float dm_pos = 0.f, dm_neg = 0.f;
+    if (DEFER == 2) {
+        dm_pos = __ldcg(a.prev_means);
+        dm_neg = -__ldcg(a.prev_means + 1);
+    }
+    // the residual owed from the previous step: x - (x >= 0 ? m_pos : -m_neg)
+    auto owed = [&](float x) { return DEFER == 2 ? x - (x >= 0.0f ? dm_pos : dm_neg) : x; };
+    auto owed_vec = [&](Vec<VW> x) {
+        if (DEFER == 2) {
+#pragma unroll
+            for (int k = 0; k < VW; ++k) x.v[k] = owed(x.v[k]);
+        }
+        return x;
+    };
     const uint64_t nv = a.n / VW;
     const uint64_t full_words = a.n >> 5;
     uint32_t *mask = MASK ? a.pos_mask + (uint64_t)p * ((a.n + 31) >> 5) : nullptr;
@@ -390,7 +415,8 @@ __global__ void __launch_bounds__(kBlock) k_encode_vec(EncodeArgs a)
         unsigned bits[U];
 #pragma unroll
         for (int u = 0; u < U; ++u) {
-            const Vec<VW> v = EF ? add_vec<VW>(gv[u], ev[u]) : gv[u];
+            const Vec<VW> v = EF ? add_vec<VW>(gv[u], owed_vec(ev[u])) : gv[u];
+            if (DEFER) st_vec<VW>(e_out + VW * (j + u * stride), v);
             split_vec<VW>(v, sp[u], sn[u], acc.n_pos, bits[u]);
         }
         acc.s_pos += (double)tree_sum<U>(sp);
@@ -404,7 +430,8 @@ __global__ void __launch_bounds__(kBlock) k_encode_vec(EncodeArgs a)
         unsigned bits = 0;
         if (j < nv) {
             Vec<VW> v = g.template vec<VW>(VW * j);
-            if (EF) v = add_vec<VW>(v, ld_vec<VW>(e + VW * j));
+            if (EF) v = add_vec<VW>(v, owed_vec(ld_vec<VW>(e + VW * j)));
+            if (DEFER) st_vec<VW>(e_out + VW * j, v);
             split_vec<VW>(v, sp, sn, acc.n_pos, bits);
         }
         acc.s_pos += (double)sp;
@@ -416,15 +443,17 @@ __global__ void __launch_bounds__(kBlock) k_encode_vec(EncodeArgs a)
         const uint64_t i = nv * VW + threadIdx.x;
         if (threadIdx.x < VW && i < a.n) {
             float v = g.one(i);
-            if (EF) v += ld_stream1(e + i);
+            if (EF) v += owed(ld_stream1(e + i));
+            if (DEFER) st_stream1(e_out + i, v);
             float sp, sn;
             unsigned bit;
             split1(v, sp, sn, acc.n_pos, bit);
             acc.s_pos += (double)sp;
             acc.s_neg += (double)sn;
         }
-        // the last, partial mask word (n % 32 elements): one warp re-reads them
-        if (MASK && threadIdx.x < 32 && (a.n & 31u)) {
+        // the last, partial mask word (n % 32 elements): one warp re-reads them.  Not in the
+        // deferred form (the buffer is being rewritten): its decode reads v itself for those elements.
+        if (MASK && !DEFER && threadIdx.x < 32 && (a.n & 31u)) {
             const uint64_t i2 = (full_words << 5) + lane;
             bool pos = false;
             if (i2 < a.n) {
@@ -756,6 +785,115 @@ __global__ void __launch_bounds__(kBlock) k_decode_scalar(DecodeArgs a)
         }
         float *wp = a.w + (int64_t)p_lo * a.w_stride + i;
         *wp = fmaf(scale, sum, *wp);
+    }
+}
+
+// ------------------------------------------------------------------ K3', deferred-residual form
+// The error buffer already holds v (written by the encode kernel) and the residual is not formed
+// until the next step, so decoding needs only pos(v) — one bit per worker-element from the packed
+// mask — and w: (P/8 + 8) bytes per model element instead of (12P + 8).  g_hat values are summed in
+// worker order exactly as in k_decode_shared_vec, so w is bit-identical to the canonical path.
+// The mask covers the full 32-element words; the last n % 32 elements are decoded from v itself.
+struct DeferredDecodeArgs {
+    float *w;
+    int64_t w_stride; // 0 = shared
+    const float *v;   // the error buffer, holding v
+    int64_t v_stride;
+    const uint32_t *mask; // [P][ceil(n/32)]
+    uint64_t n;
+    uint32_t P;
+    const float *global_means; // [2], this step's
+    float *prev_means;         // [2], out: copy of this step's means for the next encode
+    float lr;
+};
+
+template <int PT, bool REPL>
+__global__ void __launch_bounds__(kBlock) k_decode_deferred(DeferredDecodeArgs a)
+{
+    pdl_wait_prior_grid();
+    pdl_release_next_grid();
+    const uint32_t P = PT > 0 ? PT : a.P;
+    const float m_pos = __ldg(a.global_means), m_neg = __ldg(a.global_means + 1);
+    const float g_pos = m_pos, g_neg = -m_neg;
+    const float scale = REPL ? -a.lr : -a.lr / (float)P;
+    const uint64_t words = (a.n + 31) >> 5, full_words = a.n >> 5;
+    const uint64_t nv = full_words * 4; // 8-element vectors covered by full mask words
+    const uint64_t stride = (uint64_t)gridDim.x * kBlock;
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        a.prev_means[0] = m_pos;
+        a.prev_means[1] = m_neg;
+    }
+    for (uint64_t j = (uint64_t)blockIdx.x * kBlock + threadIdx.x; j < nv; j += stride) {
+        const unsigned shift = 8u * (unsigned)(j & 3);
+        if (REPL) {
+            for (uint32_t p = 0; p < P; ++p) {
+                const unsigned bits = (__ldg(a.mask + (uint64_t)p * words + (j >> 2)) >> shift) & 0xffu;
+                float *wp = a.w + (int64_t)p * a.w_stride + 8 * j;
+                Vec<8> wv = ld_vec<8>(wp);
+#pragma unroll
+                for (int k = 0; k < 8; ++k) wv.v[k] = fmaf(scale, ((bits >> k) & 1u) ? g_pos : g_neg, wv.v[k]);
+                st_vec<8>(wp, wv);
+            }
+        } else {
+            const Vec<8> wv = ld_vec<8>(a.w + 8 * j);
+            Vec<8> sum = zero_vec<8>();
+            if (PT > 0) {
+                unsigned bits[PT > 0 ? PT : 1];
+#pragma unroll
+                for (int p = 0; p < PT; ++p) bits[p] = (__ldg(a.mask + (uint64_t)p * words + (j >> 2)) >> shift) & 0xffu;
+#pragma unroll
+                for (int p = 0; p < PT; ++p) {
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) sum.v[k] += ((bits[p] >> k) & 1u) ? g_pos : g_neg;
+                }
+            } else {
+                for (uint32_t p = 0; p < P; ++p) {
+                    const unsigned bits = (__ldg(a.mask + (uint64_t)p * words + (j >> 2)) >> shift) & 0xffu;
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) sum.v[k] += ((bits >> k) & 1u) ? g_pos : g_neg;
+                }
+            }
+            st_vec<8>(a.w + 8 * j, axpy_vec<8>(scale, sum, wv));
+        }
+    }
+    // the last n % 32 elements: pos(v) read from v itself
+    if (blockIdx.x == 0 && threadIdx.x < 32) {
+        const uint64_t i = (full_words << 5) + threadIdx.x;
+        if (i < a.n) {
+            float sum = 0.f;
+            for (uint32_t p = 0; p < P; ++p) {
+                const float gh = (__ldcg(a.v + (int64_t)p * a.v_stride + i) >= 0.0f) ? g_pos : g_neg;
+                if (REPL) {
+                    float *wp = a.w + (int64_t)p * a.w_stride + i;
+                    *wp = fmaf(scale, gh, *wp);
+                } else {
+                    sum += gh;
+                }
+            }
+            if (!REPL) a.w[i] = fmaf(scale, sum, a.w[i]);
+        }
+    }
+}
+
+// Turns a buffer that holds v back into the true residual e' = v - g_hat(v) with the means of the
+// step that produced it (checkpointing, or leaving the deferred form).  grid.y = worker.
+static __global__ void __launch_bounds__(kBlock) k_materialize_err(float *v, int64_t v_stride, uint64_t n,
+                                                                   const float *means)
+{
+    pdl_wait_prior_grid();
+    pdl_release_next_grid();
+    float *row = v + (int64_t)blockIdx.y * v_stride;
+    const float g_pos = __ldg(means), g_neg = -__ldg(means + 1);
+    const uint64_t nv = n / 8, stride = (uint64_t)gridDim.x * kBlock;
+    for (uint64_t j = (uint64_t)blockIdx.x * kBlock + threadIdx.x; j < nv; j += stride) {
+        Vec<8> x = ld_vec<8>(row + 8 * j);
+#pragma unroll
+        for (int k = 0; k < 8; ++k) x.v[k] = x.v[k] - (x.v[k] >= 0.0f ? g_pos : g_neg);
+        st_vec<8>(row + 8 * j, x);
+    }
+    if (blockIdx.x == 0 && threadIdx.x < 8) {
+        const uint64_t i = nv * 8 + threadIdx.x;
+        if (i < n) row[i] = row[i] - (row[i] >= 0.0f ? g_pos : g_neg);
     }
 }
 
