@@ -200,6 +200,11 @@ int a2sgd_segments_destroy(a2sgd_segments *plan);
  * counts are left in the context for a2sgd_read_stats, as with a2sgd_step. */
 int a2sgd_step_segments(a2sgd_ctx *ctx, a2sgd_segments *plan, float lr, void *stream);
 
+/* a2sgd_step_segments with one learning rate per tensor: lr_per_segment is a DEVICE array of S
+ * floats.  This is the hook for layer-wise learning-rate policies such as LARS (listed in the
+ * paper's experimental setup for VGG-16); computing those rates is the caller's business. */
+int a2sgd_step_segments_lr(a2sgd_ctx *ctx, a2sgd_segments *plan, const float *lr_per_segment, void *stream);
+
 /* a2sgd_step for a caller whose fresh gradients sit in HOST memory (pinned
  * memory makes the copies asynchronous): copies grad_host -> grad_staging
  * worker by worker, runs the step, copies the 2P local and 2 global means

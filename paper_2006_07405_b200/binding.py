@@ -85,6 +85,8 @@ def lib() -> ctypes.CDLL:
         l.a2sgd_step_bf16.argtypes = [_vp, _vp, _i64, _vp, _i64, _vp, _i64, ctypes.c_float, _vp]
         l.a2sgd_materialize_err.restype = ctypes.c_int
         l.a2sgd_materialize_err.argtypes = [_vp, _vp, _i64, _vp]
+        l.a2sgd_step_segments_lr.restype = ctypes.c_int
+        l.a2sgd_step_segments_lr.argtypes = [_vp, _vp, _vp, _vp]
         l.a2sgd_status_string.restype = ctypes.c_char_p
         l.a2sgd_status_string.argtypes = [ctypes.c_int]
         _lib = l
@@ -304,6 +306,14 @@ def a2sgd_segments_destroy(plan: Segments) -> None:
 
 def a2sgd_step_segments(ctx: Context, plan: Segments, lr: float, stream=None) -> None:
     _check(lib().a2sgd_step_segments(ctx.handle, plan.handle, float(lr), _stream(stream)), "a2sgd_step_segments")
+
+
+def a2sgd_step_segments_lr(ctx: Context, plan: Segments, lr_per_segment: torch.Tensor, stream=None) -> None:
+    """lr_per_segment: float32 CUDA tensor of S learning rates (layer-wise policies such as LARS)."""
+    if lr_per_segment.dtype != torch.float32 or not lr_per_segment.is_cuda or not lr_per_segment.is_contiguous():
+        raise ValueError("lr_per_segment: need a contiguous float32 CUDA tensor")
+    _check(lib().a2sgd_step_segments_lr(ctx.handle, plan.handle, lr_per_segment.data_ptr(), _stream(stream)),
+           "a2sgd_step_segments_lr")
 
 
 def a2sgd_step_host(ctx: Context, w: torch.Tensor, grad_host: torch.Tensor, grad_staging: torch.Tensor,

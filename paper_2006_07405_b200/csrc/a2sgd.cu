@@ -869,7 +869,20 @@ extern "C" int a2sgd_segments_destroy(a2sgd_segments *sg)
     return A2SGD_OK;
 }
 
+static int step_segments_impl(a2sgd_ctx *c, a2sgd_segments *sg, float lr, const float *lr_per_segment, void *stream);
+
 extern "C" int a2sgd_step_segments(a2sgd_ctx *c, a2sgd_segments *sg, float lr, void *stream)
+{
+    return step_segments_impl(c, sg, lr, nullptr, stream);
+}
+
+extern "C" int a2sgd_step_segments_lr(a2sgd_ctx *c, a2sgd_segments *sg, const float *lr_per_segment, void *stream)
+{
+    if (!lr_per_segment || !aligned(lr_per_segment, 4)) return lr_per_segment ? A2SGD_ERR_ALIGN : A2SGD_ERR_ARG;
+    return step_segments_impl(c, sg, 0.0f, lr_per_segment, stream);
+}
+
+static int step_segments_impl(a2sgd_ctx *c, a2sgd_segments *sg, float lr, const float *lr_per_segment, void *stream)
 {
     if (!c || !sg || sg->ctx != c) return A2SGD_ERR_ARG;
     DeviceGuard guard(c->device);
@@ -886,6 +899,7 @@ extern "C" int a2sgd_step_segments(a2sgd_ctx *c, a2sgd_segments *sg, float lr, v
     t.w = sg->w;
     t.S = sg->S;
     t.w_replicated = sg->replicated ? 1u : 0u;
+    t.lr_per_segment = lr_per_segment;
     {
         EncodeArgs a = make_encode_args(c, nullptr, 0, nullptr, 0, c->local_means, c->pos_counts, nullptr,
                                         c->global_means);

@@ -35,6 +35,7 @@ struct SegTables {
     float *const *w;            // [S] (shared) or [P][S] (replicas)
     uint32_t S;
     uint32_t w_replicated;
+    const float *lr_per_segment; // [S] device, or nullptr: one learning rate for the whole model
 };
 
 // K1 over a segment list.  grid = (G, P); CTA x walks tiles x, x + G, ...
@@ -110,7 +111,6 @@ __global__ void __launch_bounds__(kBlock) k_decode_segments(DecodeArgs a, SegTab
     const uint32_t P = PT > 0 ? PT : a.P;
     const float m_pos = __ldg(a.global_means), m_neg = __ldg(a.global_means + 1);
     const bool repl = t.w_replicated != 0;
-    const float scale = repl ? -a.lr : -a.lr / (float)P;
     if (PT == 0) {
         for (uint32_t p = threadIdx.x; p < P; p += kBlock) sh_c[p] = worker_const<EF>(a, p, m_pos, m_neg);
         __syncthreads();
@@ -119,6 +119,9 @@ __global__ void __launch_bounds__(kBlock) k_decode_segments(DecodeArgs a, SegTab
         const SegTile d = t.tiles[tile];
         const uint64_t n_s = t.numel[d.seg];
         const uint64_t i = d.offset + (uint64_t)threadIdx.x * kSegVW;
+        // layer-wise learning rates (e.g. LARS, which the paper uses for VGG-16): one per tensor
+        const float lr = t.lr_per_segment ? __ldg(t.lr_per_segment + d.seg) : a.lr;
+        const float scale = repl ? -lr : -lr / (float)P;
         if ((d.flags & kSegFlagVec) && i + kSegVW <= n_s) {
             if (PT > 0 && !repl) {
                 constexpr int PP = PT > 0 ? PT : 1;

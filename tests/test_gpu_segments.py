@@ -113,3 +113,47 @@ def test_segment_plan_argument_checks():
         B.a2sgd_segments_create(ctx, bad, bad, w)                # sizes do not add up to n
     assert ei.value.status == B.ERR_ARG
     ctx.destroy()
+
+
+@pytest.mark.parametrize("mode", [EF, ALG1])
+@pytest.mark.parametrize("replicated", [False, True])
+def test_per_segment_learning_rates(mode, replicated):
+    """Layer-wise learning rates (the hook for LARS): the means are whole-model, the update of
+    each tensor uses its own rate.  Reference: the oracle's encode on the concatenation, then its
+    decode tensor by tensor with that tensor's rate."""
+    P = 4
+    sizes = [5, 2048, 70_001, 33, 4096, 12_345]
+    offsets = [0, 0, 1, 0]
+    n = sum(sizes)
+    gen = torch.Generator("cuda").manual_seed(77)
+    grad = [_tensors(sizes, offsets, gen, 1e-3) for _ in range(P)]
+    err = [_tensors(sizes, offsets, gen, 3e-4) for _ in range(P)]
+    w = [_tensors(sizes, offsets, gen, 0.02) for _ in range(P if replicated else 1)]
+    lrs = np.array([0.5, 0.01, 0.2, 1.0, 0.05, 0.125], np.float32)
+    gh, eh = _cat(grad), _cat(err)
+    wh = _cat(w) if replicated else _cat(w)[0]
+    lm_ref, cnt_ref, _ = oracle.encode(gh, eh if mode == EF else None, mode=mode)
+    gm_ref = oracle.global_average(lm_ref)
+    off = 0
+    for s, lr in zip(sizes, lrs):
+        g_s = np.ascontiguousarray(gh[:, off:off + s])
+        e_s = np.ascontiguousarray(eh[:, off:off + s])
+        w_s = np.ascontiguousarray(wh[:, off:off + s]) if replicated else wh[off:off + s].copy()
+        oracle.decode_update(w_s, g_s, e_s, lm_ref, gm_ref, float(lr), mode=mode)
+        eh[:, off:off + s] = e_s
+        if replicated:
+            wh[:, off:off + s] = w_s
+        else:
+            wh[off:off + s] = w_s
+        off += s
+    ctx = B.a2sgd_create(n, P, 0, mode)
+    plan = B.a2sgd_segments_create(ctx, grad, err, w if replicated else w[0], w_replicated=replicated)
+    B.a2sgd_step_segments_lr(ctx, plan, torch.from_numpy(lrs).cuda())
+    lm, gm, cnt, status = B.a2sgd_read_stats(ctx)
+    assert status == B.OK and np.array_equal(cnt, cnt_ref)
+    assert_means(lm, lm_ref)
+    assert_means(gm, gm_ref)
+    w_got = _cat(w) if replicated else _cat(w)[0]
+    assert_state(w_got, wh, _cat(err), eh, gm_ref, "per-segment lr")
+    plan.destroy()
+    ctx.destroy()
