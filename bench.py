@@ -186,6 +186,52 @@ def run_reference(args):
     print(json.dumps(line), flush=True)
 
 
+# ----------------------------------------------------------------------------- profiler helper
+def run_variant(wl, variant, steps, warmup, dev):
+    """--minimal --variant X: a bare loop of one entry point, for profiler captures of the kernels
+    the plain step loop does not launch.  Returns ms per call."""
+    import torch
+    from paper_2006_07405_b200 import binding as B
+    from paper_2006_07405_b200 import workloads as W
+    n, P = wl.n, wl.P
+    g = B.padded_rows(P, n, dev)
+    e = B.padded_rows(P, n, dev, fill=0.0)
+    w = torch.empty(n, device=dev)
+    W.fill_gradients(wl, 0, g)
+    W.init_weights(wl, w)
+    flags = B.MODE_EF
+    if variant == "deferred":
+        flags |= B.DEFERRED_RESIDUAL
+    elif variant == "single_launch":
+        flags |= B.FORCE_COOPERATIVE
+    ctx = B.a2sgd_create(n, P, dev.index, flags)
+    if variant == "dense_sync":
+        call = lambda: B.a2sgd_dense_sync(ctx, w, g, wl.lr)
+    elif variant == "bf16":
+        g16 = torch.empty((P, g.stride(0)), dtype=torch.bfloat16, device=dev)[:, :n]
+        g16.copy_(g)
+        call = lambda: B.a2sgd_step_bf16(ctx, w, g16, e, wl.lr)
+    elif variant == "segments":
+        sizes = [sg.numel for sg in wl.segments]
+        gs = [[t.clone() for t in torch.split(g[p], sizes)] for p in range(P)]
+        es = [[t.clone() for t in torch.split(e[p], sizes)] for p in range(P)]
+        ws = [t.clone() for t in torch.split(w, sizes)]
+        plan = B.a2sgd_segments_create(ctx, gs, es, ws)
+        call = lambda: B.a2sgd_step_segments(ctx, plan, wl.lr)
+    else:  # deferred, single_launch: the step entry point of a context created with that flag
+        call = lambda: B.a2sgd_step(ctx, w, g, e, wl.lr)
+    for _ in range(max(3, warmup)):
+        call()
+    torch.cuda.synchronize(dev)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record()
+    for _ in range(steps):
+        call()
+    ev1.record()
+    torch.cuda.synchronize(dev)
+    return ev0.elapsed_time(ev1) / steps
+
+
 # ----------------------------------------------------------------------------- device arm
 def max_over_ranks(ms: float, dist, device) -> float:
     """Every rank contributes its own device-timed milliseconds; all get the maximum."""
@@ -419,6 +465,9 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--scale-div", type=int, default=1,
                     help="divide every tensor length of the workload (small cases for profiler captures)")
+    ap.add_argument("--variant", default="step",
+                    choices=["step", "dense_sync", "deferred", "bf16", "segments", "single_launch"],
+                    help="with --minimal: which entry point the bare loop calls")
     ap.add_argument("--minimal", action="store_true",
                     help="timed step loop only (for profiler captures): no e2e, no per-kernel loop, "
                          "no extra workloads, no clock load loop, no CPU baseline")
@@ -454,6 +503,11 @@ def main():
     peak_gbs, peak_src = measured_peak_gbs()
     steps, warmup = max(1, args.steps), max(3, args.warmup)
 
+    if args.minimal and args.variant != "step":
+        ms = run_variant(wl, args.variant, steps, warmup, dev)
+        print(json.dumps({"variant": args.variant, "ms_per_call": ms, "steps": steps, "config": W.describe(wl),
+                          "note": "minimal run for profiler captures"}), flush=True)
+        return
     if args.minimal:
         res = time_workload(wl, steps, warmup, dev, with_roofline=False, with_e2e=False, dist=dist)
         if rank == 0:
