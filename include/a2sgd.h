@@ -92,7 +92,9 @@ enum a2sgd_flags {
                                          of 8 (A2SGD_ERR_ALIGN otherwise), the same error buffer at every
                                          step, and only a2sgd_step / a2sgd_step_host / a2sgd_dense_sync /
                                          a2sgd_materialize_err on this context.  The context also owns a sign
-                                         mask of P*n/8 bytes. */
+                                         mask of P*n/8 bytes.  Which kernel a step launches depends on
+                                         host-side state (does the buffer hold v yet?), so a captured step
+                                         must not be replayed across the first step or a materialise call. */
     A2SGD_TEST_BARRIER_NEVER_OPENS = 1 << 9 /* test hook: the single-launch path waits for one arrival more
                                                than its grid has, with a ~0.2 ms limit, so every CTA gives up,
                                                writes nothing and A2SGD_ERR_TIMEOUT is latched */

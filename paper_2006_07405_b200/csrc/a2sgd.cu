@@ -53,9 +53,8 @@ struct a2sgd_ctx {
     float *global_means = nullptr;
     unsigned long long *pos_counts = nullptr;
     unsigned int *tickets = nullptr;
-    unsigned int *barrier = nullptr; // 2 words: arrival counter, release epoch
+    unsigned int *barrier = nullptr; // 2 words: arrival counter, generation counter
     int *status = nullptr;
-    unsigned int coop_epoch = 0;
     // deferred-residual representation (A2SGD_DEFERRED_RESIDUAL)
     uint32_t *sign_mask = nullptr; // [P][ceil(n/32)]
     float *prev_means = nullptr;   // [2]
@@ -460,9 +459,6 @@ int launch_coop(a2sgd_ctx *c, const void *fn, uint32_t grid, float *w, int64_t w
     a.enc = make_encode_args(c, grad, gs, err, es, c->local_means, c->pos_counts, nullptr, c->global_means);
     a.dec = make_decode_args(c, w, ws, grad, gs, err, es, c->local_means, c->global_means, lr);
     a.barrier = c->barrier;
-    c->coop_epoch += 1;
-    if (c->coop_epoch == 0) c->coop_epoch = 1;
-    a.epoch = c->coop_epoch;
     const bool never_opens = (c->flags & A2SGD_TEST_BARRIER_NEVER_OPENS) != 0;
     a.expected = never_opens ? grid + 1 : grid;
     a.spin_limit = never_opens ? (1u << 12) : (1u << 24); // x 40 ns sleep: ~0.2 ms / ~1 s

@@ -985,8 +985,7 @@ __global__ void __launch_bounds__(kBlock) static k_dense_sync_scalar(DenseArgs a
 struct CoopArgs {
     EncodeArgs enc;            // pos_mask unused; global_means required
     DecodeArgs dec;
-    unsigned int *barrier;     // [0] arrival counter (zero between launches), [1] release epoch
-    unsigned int epoch;        // value that opens the barrier for this launch (never 0)
+    unsigned int *barrier;     // [0] arrival counter (zero between launches), [1] generation counter
     unsigned int expected;     // arrivals that open the barrier (= gridDim.x in normal use)
     unsigned int spin_limit;   // polls before giving up
 };
@@ -1010,6 +1009,7 @@ struct CoopShared {
     double part[PT][2][kWarps];
     unsigned long long cnt[PT][kWarps];
     float mu[PT][2];
+    unsigned int generation;
     int flag;
 };
 
@@ -1060,7 +1060,12 @@ __device__ __forceinline__ bool coop_reduce_and_barrier(const CoopArgs &a, Acc (
     }
     __syncthreads();
     // ---- grid barrier (one fence per CTA: fences are the expensive part of this path)
+    // The release word is a generation counter that lives on the device: every CTA notes its value
+    // before arriving and waits for it to change; the last arriver increments it.  It cannot change
+    // before all CTAs have arrived, hence after all have read it.  Nothing depends on a value passed
+    // from the host, so a captured launch can be replayed any number of times.
     if (threadIdx.x == 0) {
+        sh.generation = ld_acquire_u32(&a.barrier[1]);
         __threadfence();
         const unsigned int t = atomicAdd(&a.barrier[0], 1u);
         sh.flag = (t == a.expected - 1) ? 1 : 0;
@@ -1118,14 +1123,14 @@ __device__ __forceinline__ bool coop_reduce_and_barrier(const CoopArgs &a, Acc (
             ea.global_means[1] = (float)(gn / (double)PT);
             a.barrier[0] = 0;
             __threadfence();
-            st_release_u32(&a.barrier[1], a.epoch);
+            st_release_u32(&a.barrier[1], sh.generation + 1u);
         }
         __syncthreads();
     } else {
         if (threadIdx.x == 0) {
             unsigned int polls = 0;
             int ok = 1;
-            while (ld_acquire_u32(&a.barrier[1]) != a.epoch) {
+            while (ld_acquire_u32(&a.barrier[1]) == sh.generation) {
                 if (++polls > a.spin_limit) {
                     ok = 0;
                     break;

@@ -630,3 +630,39 @@ def test_two_contexts_on_two_streams_do_not_interfere():
         assert status == B.OK
         assert_state(w.cpu().numpy(), refs[k][1], e.cpu().numpy(), refs[k][0], gm, f"stream {k}", max_outliers=2)
         ctx.destroy()
+
+
+def test_single_launch_step_replayed_from_a_one_step_graph():
+    """A graph holding ONE cooperative step, replayed several times: the grid barrier must not
+    depend on anything fixed at capture time."""
+    n, P = 300_000, 1
+    gen = torch.Generator("cuda").manual_seed(5)
+    g = B.padded_rows(P, n, "cuda"); g.normal_(0.0, 1e-3, generator=gen)
+    e0 = B.padded_rows(P, n, "cuda"); e0.normal_(0.0, 1e-4, generator=gen)
+    w0 = torch.randn(n, device="cuda", generator=gen) * 0.02
+
+    def run(use_graph):
+        e = B.padded_rows(P, n, "cuda"); e.copy_(e0)
+        w = w0.clone()
+        ctx = B.a2sgd_create(n, P, 0, EF | B.FORCE_COOPERATIVE)
+        B.a2sgd_step(ctx, w, g, e, 0.1)
+        if use_graph:
+            side = torch.cuda.Stream()
+            side.wait_stream(torch.cuda.current_stream())
+            with torch.cuda.stream(side):
+                graph = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(graph, stream=side):
+                    B.a2sgd_step(ctx, w, g, e, 0.1, stream=side)
+            torch.cuda.current_stream().wait_stream(side)
+            for _ in range(4):
+                graph.replay()
+        else:
+            for _ in range(4):
+                B.a2sgd_step(ctx, w, g, e, 0.1)
+        lm, gm, cnt, status = B.a2sgd_read_stats(ctx)
+        out = (status, lm.tobytes(), gm.tobytes(), cnt.tobytes(), w.cpu().numpy().tobytes(), e.cpu().numpy().tobytes())
+        ctx.destroy()
+        return out
+
+    eager, replayed = run(False), run(True)
+    assert eager[0] == B.OK and eager == replayed
