@@ -483,7 +483,9 @@ def main():
 
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the A2SGD path has no CPU fallback")
-    B.lib()  # fail loudly if the CUDA library has not been built
+    from paper_2006_07405_b200 import build as cuda_build
+    cuda_build.build()   # compiles only when the library is missing or older than its sources (atomic replace)
+    B.lib()  # fails loudly if the CUDA library is still missing: there is no other path
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))

@@ -25,3 +25,13 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+@pytest.fixture(scope="session", autouse=True)
+def _native_libraries_built():
+    """Compile the CUDA library (nvcc) and the C oracle (gcc) if they are missing or stale, so
+    that the tests always run against the sources in the tree."""
+    from paper_2006_07405_b200 import build as cuda_build
+    import oracle
+    cuda_build.build()
+    oracle.build()
