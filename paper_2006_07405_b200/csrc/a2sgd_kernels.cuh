@@ -295,44 +295,71 @@ __device__ __forceinline__ void finish_worker(const EncodeArgs &a, uint32_t p, d
     __syncthreads();
     if (*sh_flag == 0) return;
     __threadfence();
-    // last CTA of this worker: fold the G partials, thread t takes t, t+kBlock, ... in order
+    // last CTA of this worker: fold the G partials, thread t takes t, t+kBlock, ... in order.
+    // The loads of a batch are issued together (one L2 round trip per four partials, not four);
+    // the additions stay in index order.
     double fp = 0.0, fn = 0.0;
     unsigned long long fc = 0;
-    for (uint32_t i = threadIdx.x; i < G; i += kBlock) {
-        fp += __ldcg(&mine[i].s_pos);
-        fn += __ldcg(&mine[i].s_neg);
-        fc += __ldcg(&mine[i].n_pos);
+    for (uint32_t base = threadIdx.x; base < G; base += 4 * kBlock) {
+        double bp[4], bn[4];
+        unsigned long long bc[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const uint32_t i = base + u * kBlock;
+            bp[u] = i < G ? __ldcg(&mine[i].s_pos) : 0.0;
+            bn[u] = i < G ? __ldcg(&mine[i].s_neg) : 0.0;
+            bc[u] = i < G ? __ldcg(&mine[i].n_pos) : 0ull;
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            fp += bp[u];
+            fn += bn[u];
+            fc += bc[u];
+        }
     }
     __syncthreads();
     block_reduce(fp, fn, fc, sh_d, sh_n);
-    if (threadIdx.x != 0) return;
-    const unsigned long long n_neg = a.n - fc;
-    const float mu_pos = fc ? (float)(fp / (double)fc) : 0.0f;
-    const float mu_neg = n_neg ? (float)(fn / (double)n_neg) : 0.0f;
-    if (!isfinite(fp) || !isfinite(fn)) atomicCAS(a.status, kDevOk, kDevNonFinite);
-    a.local_means[2 * p + 0] = mu_pos;
-    a.local_means[2 * p + 1] = mu_neg;
-    if (a.pos_counts) a.pos_counts[p] = fc;
-    if (a.ctx_local_means && a.ctx_local_means != a.local_means) {
-        a.ctx_local_means[2 * p + 0] = mu_pos;
-        a.ctx_local_means[2 * p + 1] = mu_neg;
-    }
-    if (a.ctx_pos_counts && a.ctx_pos_counts != a.pos_counts) a.ctx_pos_counts[p] = fc;
-    a.tickets[p] = 0; // ready for the next launch
-    if (a.global_means) {
-        __threadfence();
-        const unsigned int t = atomicAdd(&a.tickets[a.P], 1u);
-        if (t == a.P - 1) {
-            __threadfence();
-            double gp = 0.0, gn = 0.0;
-            for (uint32_t q = 0; q < a.P; ++q) { // worker order
-                gp += (double)__ldcg(&a.local_means[2 * q + 0]);
-                gn += (double)__ldcg(&a.local_means[2 * q + 1]);
-            }
-            a.global_means[0] = (float)(gp / (double)a.P);
-            a.global_means[1] = (float)(gn / (double)a.P);
-            a.tickets[a.P] = 0;
+    if (threadIdx.x == 0) {
+        const unsigned long long n_neg = a.n - fc;
+        const float mu_pos = fc ? (float)(fp / (double)fc) : 0.0f;
+        const float mu_neg = n_neg ? (float)(fn / (double)n_neg) : 0.0f;
+        if (!isfinite(fp) || !isfinite(fn)) atomicCAS(a.status, kDevOk, kDevNonFinite);
+        a.local_means[2 * p + 0] = mu_pos;
+        a.local_means[2 * p + 1] = mu_neg;
+        if (a.pos_counts) a.pos_counts[p] = fc;
+        if (a.ctx_local_means && a.ctx_local_means != a.local_means) {
+            a.ctx_local_means[2 * p + 0] = mu_pos;
+            a.ctx_local_means[2 * p + 1] = mu_neg;
         }
+        if (a.ctx_pos_counts && a.ctx_pos_counts != a.pos_counts) a.ctx_pos_counts[p] = fc;
+        a.tickets[p] = 0; // ready for the next launch
+        int last_of_all = 0;
+        if (a.global_means) {
+            __threadfence();
+            last_of_all = atomicAdd(&a.tickets[a.P], 1u) == a.P - 1 ? 1 : 0;
+        }
+        *sh_flag = last_of_all;
+    }
+    __syncthreads();
+    if (*sh_flag == 0) return;
+    // The CTA that finished the last worker averages the 2P scalars (Algorithm 1 line 5).  The
+    // loads are spread over the CTA (P can be 1024); the sum itself runs in worker order in fp64.
+    __threadfence();
+    __shared__ float sh_mu[2][kMaxP];
+    for (uint32_t q = threadIdx.x; q < a.P; q += kBlock) {
+        sh_mu[0][q] = __ldcg(&a.local_means[2 * q + 0]);
+        sh_mu[1][q] = __ldcg(&a.local_means[2 * q + 1]);
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        double gp = 0.0, gn = 0.0;
+        for (uint32_t q = 0; q < a.P; ++q) { // worker order
+            gp += (double)sh_mu[0][q];
+            gn += (double)sh_mu[1][q];
+        }
+        a.global_means[0] = (float)(gp / (double)a.P);
+        a.global_means[1] = (float)(gn / (double)a.P);
+        a.tickets[a.P] = 0;
     }
 }
 
