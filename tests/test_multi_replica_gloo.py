@@ -64,3 +64,17 @@ def test_single_rank_passthrough():
     assert bench.algorithmic_bytes_per_model_element(4) == {"encode": 32, "decode": 56, "step": 88}
     assert bench.algorithmic_bytes_per_model_element(8)["step"] == 168
     assert bench.algorithmic_bytes_per_model_element(1)["step"] == 28
+
+
+def test_reference_arm_json_line_has_the_contract_keys():
+    import json
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--workload",
+                          "c1_flat_1m", "--steps", "2", "--warmup", "1"], capture_output=True, text=True, timeout=600)
+    assert out.returncode == 0, out.stderr
+    line = json.loads(out.stdout.strip().splitlines()[-1])
+    for key in ("impl", "metric", "value", "unit", "n_gpus", "steps", "warmup", "ms_per_step", "higher_is_better",
+                "scaling", "vs_baseline", "dtype", "data", "config", "cpu_baseline", "e2e"):
+        assert key in line, key
+    assert line["impl"] == "reference" and line["cpu_baseline"]["kind"] == "oracle" and line["cpu_baseline"]["cores"] == 1
+    assert line["e2e"]["h2d_bytes_per_step"] == 0 and line["e2e"]["d2h_bytes_per_step"] == 0
+    assert line["value"] > 0 and line["config"]["workload"] == "c1_flat_1m"
