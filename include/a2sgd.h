@@ -95,6 +95,11 @@ enum a2sgd_flags {
                                          mask of P*n/8 bytes.  Which kernel a step launches depends on
                                          host-side state (does the buffer hold v yet?), so a captured step
                                          must not be replayed across the first step or a materialise call. */
+    A2SGD_CHECK_POINTERS = 1 << 8,    /* every call first asks the runtime whether each buffer is device (or
+                                         managed) memory usable from the context's device and returns
+                                         A2SGD_ERR_ARG otherwise, before anything is launched: a host pointer
+                                         handed to a kernel would fault the GPU.  Costs about a microsecond
+                                         per pointer per call; off by default. */
     A2SGD_TEST_BARRIER_NEVER_OPENS = 1 << 9 /* test hook: the single-launch path waits for one arrival more
                                                than its grid has, with a ~0.2 ms limit, so every CTA gives up,
                                                writes nothing and A2SGD_ERR_TIMEOUT is latched */

@@ -24,6 +24,7 @@ MODE_ALG1 = 1
 FORCE_TWO_PASS = 1 << 4
 FORCE_COOPERATIVE = 1 << 5
 DEFERRED_RESIDUAL = 1 << 7
+CHECK_POINTERS = 1 << 8
 TEST_BARRIER_NEVER_OPENS = 1 << 9
 ROW_ALIGN_ELEMS = 32   # 128 bytes: rows that start on a cache-line boundary take the widest vector kernels
 

@@ -517,10 +517,24 @@ int deferred_step(a2sgd_ctx *c, float *w, int64_t ws, const float *grad, int64_t
     return A2SGD_OK;
 }
 
+// A2SGD_CHECK_POINTERS: is this address device (or managed) memory that the context's device can use?
+bool device_pointer_ok(const a2sgd_ctx *c, const void *p)
+{
+    if (!(c->flags & A2SGD_CHECK_POINTERS) || p == nullptr) return true;
+    cudaPointerAttributes attr{};
+    if (cudaPointerGetAttributes(&attr, p) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return false;
+    }
+    if (attr.type == cudaMemoryTypeManaged) return true;
+    return attr.type == cudaMemoryTypeDevice && attr.device == c->device;
+}
+
 int check_common(const a2sgd_ctx *c, const float *grad, int64_t gs, const float *err, int64_t es,
                  bool err_required)
 {
     if (!c || !grad) return A2SGD_ERR_ARG;
+    if (!device_pointer_ok(c, grad) || !device_pointer_ok(c, err)) return A2SGD_ERR_ARG;
     if (err_required && !err) return A2SGD_ERR_ARG;
     if (!stride_ok(gs, c->n, c->P)) return A2SGD_ERR_ARG;
     if (err && !stride_ok(es, c->n, c->P)) return A2SGD_ERR_ARG;
@@ -536,7 +550,7 @@ extern "C" int a2sgd_create(a2sgd_ctx **out, uint64_t n, uint32_t P, int device,
     if (!out) return A2SGD_ERR_ARG;
     *out = nullptr;
     const uint32_t known = A2SGD_MODE_ALG1 | A2SGD_FORCE_TWO_PASS | A2SGD_FORCE_COOPERATIVE |
-                           A2SGD_TEST_BARRIER_NEVER_OPENS | A2SGD_DEFERRED_RESIDUAL;
+                           A2SGD_TEST_BARRIER_NEVER_OPENS | A2SGD_DEFERRED_RESIDUAL | A2SGD_CHECK_POINTERS;
     if ((flags & A2SGD_DEFERRED_RESIDUAL) && (flags & (A2SGD_MODE_ALG1 | A2SGD_FORCE_COOPERATIVE))) return A2SGD_ERR_ARG;
     if (n == 0 || n >= (1ull << 40) || P == 0 || P > (uint32_t)kMaxP || (flags & ~known)) return A2SGD_ERR_ARG;
     if ((flags & A2SGD_FORCE_TWO_PASS) && (flags & A2SGD_FORCE_COOPERATIVE)) return A2SGD_ERR_ARG;
@@ -625,6 +639,8 @@ extern "C" int a2sgd_encode(a2sgd_ctx *c, const float *grad, int64_t grad_stride
     if (rc) return rc;
     if (!aligned(local_means, 4) || (pos_counts && !aligned(pos_counts, 8)) || (pos_mask && !aligned(pos_mask, 4)))
         return A2SGD_ERR_ALIGN;
+    if (!device_pointer_ok(c, local_means) || !device_pointer_ok(c, pos_counts) || !device_pointer_ok(c, pos_mask))
+        return A2SGD_ERR_ARG;
     DeviceGuard guard(c->device);
     if (!guard.ok) return A2SGD_ERR_CUDA;
     return launch_encode(c, grad, grad_stride, err, err_stride, local_means,
@@ -657,6 +673,8 @@ extern "C" int a2sgd_decode_update(a2sgd_ctx *c, float *w, int64_t w_stride, con
     if (w_stride != 0 && !stride_ok(w_stride, c->n, c->P)) return A2SGD_ERR_ARG;
     if (!aligned(w, 4) || !aligned(global_means, 4) || (local_means && !aligned(local_means, 4)))
         return A2SGD_ERR_ALIGN;
+    if (!device_pointer_ok(c, w) || !device_pointer_ok(c, global_means) || !device_pointer_ok(c, local_means))
+        return A2SGD_ERR_ARG;
     DeviceGuard guard(c->device);
     if (!guard.ok) return A2SGD_ERR_CUDA;
     return launch_decode(c, w, (c->P == 1) ? 0 : w_stride, grad, grad_stride, err, err_stride, local_means,
@@ -671,6 +689,7 @@ extern "C" int a2sgd_step(a2sgd_ctx *c, float *w, int64_t w_stride, const float 
     if (rc) return rc;
     if (w_stride != 0 && !stride_ok(w_stride, c->n, c->P)) return A2SGD_ERR_ARG;
     if (!aligned(w, 4)) return A2SGD_ERR_ALIGN;
+    if (!device_pointer_ok(c, w)) return A2SGD_ERR_ARG;
     DeviceGuard guard(c->device);
     if (!guard.ok) return A2SGD_ERR_CUDA;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
@@ -755,6 +774,7 @@ extern "C" int a2sgd_dense_sync(a2sgd_ctx *c, float *w, int64_t w_stride, const 
     if (!stride_ok(grad_stride, c->n, c->P)) return A2SGD_ERR_ARG;
     if (w_stride != 0 && !stride_ok(w_stride, c->n, c->P)) return A2SGD_ERR_ARG;
     if (!aligned(w, 4) || !aligned(grad, 4)) return A2SGD_ERR_ALIGN;
+    if (!device_pointer_ok(c, w) || !device_pointer_ok(c, grad)) return A2SGD_ERR_ARG;
     DeviceGuard guard(c->device);
     if (!guard.ok) return A2SGD_ERR_CUDA;
     const int64_t ws = (c->P == 1) ? 0 : w_stride;

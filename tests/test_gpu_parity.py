@@ -666,3 +666,22 @@ def test_single_launch_step_replayed_from_a_one_step_graph():
 
     eager, replayed = run(False), run(True)
     assert eager[0] == B.OK and eager == replayed
+
+
+def test_pointer_check_flag_rejects_host_memory_before_any_launch():
+    """With A2SGD_CHECK_POINTERS a host address is refused on the host; nothing reaches the GPU."""
+    n, P = 4096, 2
+    g = B.padded_rows(P, n, "cuda", 0.0)
+    e = B.padded_rows(P, n, "cuda", 0.0)
+    w = torch.zeros(n, device="cuda")
+    host = np.zeros((P, n), np.float32)
+    ctx = B.a2sgd_create(n, P, 0, EF | B.CHECK_POINTERS)
+    h = ctx.handle
+    lib = B.lib()
+    assert lib.a2sgd_step(h, w.data_ptr(), 0, host.ctypes.data, n, e.data_ptr(), e.stride(0), 0.1, None) == B.ERR_ARG
+    assert lib.a2sgd_step(h, host.ctypes.data, 0, g.data_ptr(), g.stride(0), e.data_ptr(), e.stride(0), 0.1, None) == B.ERR_ARG
+    assert lib.a2sgd_dense_sync(h, w.data_ptr(), 0, host.ctypes.data, n, 0.1, None) == B.ERR_ARG
+    B.a2sgd_step(ctx, w, g, e, 0.1)                          # device buffers pass
+    *_, status = B.a2sgd_read_stats(ctx)
+    assert status == B.OK
+    ctx.destroy()
