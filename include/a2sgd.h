@@ -164,6 +164,11 @@ int a2sgd_step_bf16(a2sgd_ctx *ctx, float *w, int64_t w_stride,
                     const uint16_t *grad, int64_t grad_stride,
                     float *err, int64_t err_stride, float lr, void *stream);
 
+/* The same with IEEE half-precision (fp16) gradients; widening is exact here too. */
+int a2sgd_step_f16(a2sgd_ctx *ctx, float *w, int64_t w_stride,
+                   const uint16_t *grad, int64_t grad_stride,
+                   float *err, int64_t err_stride, float lr, void *stream);
+
 /* For contexts created with A2SGD_DEFERRED_RESIDUAL: rewrites the error buffer in place from the
  * compensated vector v it holds after a step to the true residual e = v - g_hat(v) of that step
  * (one pass, 8 bytes per worker-element), e.g. before a checkpoint or before handing the buffer

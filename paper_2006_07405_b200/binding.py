@@ -82,8 +82,9 @@ def lib() -> ctypes.CDLL:
         l.a2sgd_segments_destroy.argtypes = [_vp]
         l.a2sgd_step_segments.restype = ctypes.c_int
         l.a2sgd_step_segments.argtypes = [_vp, _vp, ctypes.c_float, _vp]
-        l.a2sgd_step_bf16.restype = ctypes.c_int
-        l.a2sgd_step_bf16.argtypes = [_vp, _vp, _i64, _vp, _i64, _vp, _i64, ctypes.c_float, _vp]
+        for fn in (l.a2sgd_step_bf16, l.a2sgd_step_f16):
+            fn.restype = ctypes.c_int
+            fn.argtypes = [_vp, _vp, _i64, _vp, _i64, _vp, _i64, ctypes.c_float, _vp]
         l.a2sgd_materialize_err.restype = ctypes.c_int
         l.a2sgd_materialize_err.argtypes = [_vp, _vp, _i64, _vp]
         l.a2sgd_step_segments_lr.restype = ctypes.c_int
@@ -243,6 +244,17 @@ def a2sgd_materialize_err(ctx: Context, err: torch.Tensor, stream=None) -> None:
     """Deferred-residual contexts: turn the buffer (holding v) back into the true residual, in place."""
     ep, es = _rows(err, "err")
     _check(lib().a2sgd_materialize_err(ctx.handle, ep, es, _stream(stream)), "a2sgd_materialize_err")
+
+
+def a2sgd_step_f16(ctx: Context, w: torch.Tensor, grad: torch.Tensor, err: Optional[torch.Tensor], lr: float,
+                   stream=None) -> None:
+    """a2sgd_step with half-precision gradients: grad is a torch.float16 CUDA tensor [P, >= n]."""
+    if grad.dtype != torch.float16 or not grad.is_cuda or grad.dim() != 2 or (grad.shape[1] > 1 and grad.stride(1) != 1):
+        raise ValueError("grad: need a float16 CUDA tensor [P, n] with unit inner stride")
+    wp, ws = _weights(w)
+    ep, es = _rows(err, "err")
+    _check(lib().a2sgd_step_f16(ctx.handle, wp, ws, grad.data_ptr(), grad.stride(0), ep, es, float(lr),
+                                _stream(stream)), "a2sgd_step_f16")
 
 
 def a2sgd_dense_sync(ctx: Context, w: torch.Tensor, grad: torch.Tensor, lr: float, stream=None) -> None:

@@ -219,40 +219,42 @@ const void *select_decode_scalar(bool ef, bool store)
     return store ? (const void *)k_decode_scalar<false, true> : (const void *)k_decode_scalar<false, false>;
 }
 
-// bfloat16 gradient rows: 8-element (128-bit) vectors or scalar accesses
-template <bool EF, bool STORE>
-const void *select_decode_shared_bf16_p(uint32_t P)
+// 16-bit gradient rows (GT = 1 bfloat16, 2 half): 8-element (128-bit) vectors or scalar accesses
+template <bool EF, bool STORE, int GT>
+const void *select_decode_shared_lowp_p(uint32_t P)
 {
     switch (P) {
-    case 1: return (const void *)k_decode_shared_vec<EF, STORE, 1, 8, true>;
-    case 2: return (const void *)k_decode_shared_vec<EF, STORE, 2, 8, true>;
-    case 4: return (const void *)k_decode_shared_vec<EF, STORE, 4, 8, true>;
-    case 8: return (const void *)k_decode_shared_vec<EF, STORE, 8, 8, true>;
-    default: return (const void *)k_decode_shared_vec<EF, STORE, 0, 8, true>;
+    case 1: return (const void *)k_decode_shared_vec<EF, STORE, 1, 8, GT>;
+    case 2: return (const void *)k_decode_shared_vec<EF, STORE, 2, 8, GT>;
+    case 4: return (const void *)k_decode_shared_vec<EF, STORE, 4, 8, GT>;
+    case 8: return (const void *)k_decode_shared_vec<EF, STORE, 8, 8, GT>;
+    default: return (const void *)k_decode_shared_vec<EF, STORE, 0, 8, GT>;
     }
 }
 
-const void *select_encode_bf16(bool ef, int vw)
+template <int GT>
+const void *select_encode_lowp(bool ef, int vw)
 {
-    if (vw == 8) return ef ? (const void *)k_encode_vec<true, false, 8, true> : (const void *)k_encode_vec<false, false, 8, true>;
-    return ef ? (const void *)k_encode_scalar<true, false, true> : (const void *)k_encode_scalar<false, false, true>;
+    if (vw == 8) return ef ? (const void *)k_encode_vec<true, false, 8, GT> : (const void *)k_encode_vec<false, false, 8, GT>;
+    return ef ? (const void *)k_encode_scalar<true, false, GT> : (const void *)k_encode_scalar<false, false, GT>;
 }
 
-const void *select_decode_bf16(bool ef, bool store, bool shared, uint32_t P, int vw)
+template <int GT>
+const void *select_decode_lowp(bool ef, bool store, bool shared, uint32_t P, int vw)
 {
     if (vw == 8 && shared) {
-        if (ef) return select_decode_shared_bf16_p<true, true>(P);
-        return store ? select_decode_shared_bf16_p<false, true>(P) : select_decode_shared_bf16_p<false, false>(P);
+        if (ef) return select_decode_shared_lowp_p<true, true, GT>(P);
+        return store ? select_decode_shared_lowp_p<false, true, GT>(P) : select_decode_shared_lowp_p<false, false, GT>(P);
     }
     if (vw == 8) {
-        if (ef) return (const void *)k_decode_repl_vec<true, true, 8, true>;
-        return store ? (const void *)k_decode_repl_vec<false, true, 8, true> : (const void *)k_decode_repl_vec<false, false, 8, true>;
+        if (ef) return (const void *)k_decode_repl_vec<true, true, 8, GT>;
+        return store ? (const void *)k_decode_repl_vec<false, true, 8, GT> : (const void *)k_decode_repl_vec<false, false, 8, GT>;
     }
-    if (ef) return (const void *)k_decode_scalar<true, true, true>;
-    return store ? (const void *)k_decode_scalar<false, true, true> : (const void *)k_decode_scalar<false, false, true>;
+    if (ef) return (const void *)k_decode_scalar<true, true, GT>;
+    return store ? (const void *)k_decode_scalar<false, true, GT> : (const void *)k_decode_scalar<false, false, GT>;
 }
 
-// a bfloat16 row allows 8-element vectors when it is 16-byte aligned with a stride multiple of 8
+// a 16-bit row allows 8-element vectors when it is 16-byte aligned with a stride multiple of 8
 inline int vec_width_bf16(const void *p, int64_t stride, uint32_t P)
 {
     return (aligned(p, 16) && (P == 1 || stride % 8 == 0)) ? 8 : 0;
@@ -709,8 +711,23 @@ extern "C" int a2sgd_step(a2sgd_ctx *c, float *w, int64_t w_stride, const float 
     return launch_decode(c, w, ws, grad, grad_stride, err, err_stride, c->local_means, c->global_means, lr, s);
 }
 
+static int step_lowp(a2sgd_ctx *c, float *w, int64_t w_stride, const uint16_t *grad, int64_t grad_stride,
+                     float *err, int64_t err_stride, float lr, void *stream, int gt);
+
 extern "C" int a2sgd_step_bf16(a2sgd_ctx *c, float *w, int64_t w_stride, const uint16_t *grad, int64_t grad_stride,
                                float *err, int64_t err_stride, float lr, void *stream)
+{
+    return step_lowp(c, w, w_stride, grad, grad_stride, err, err_stride, lr, stream, 1);
+}
+
+extern "C" int a2sgd_step_f16(a2sgd_ctx *c, float *w, int64_t w_stride, const uint16_t *grad, int64_t grad_stride,
+                              float *err, int64_t err_stride, float lr, void *stream)
+{
+    return step_lowp(c, w, w_stride, grad, grad_stride, err, err_stride, lr, stream, 2);
+}
+
+static int step_lowp(a2sgd_ctx *c, float *w, int64_t w_stride, const uint16_t *grad, int64_t grad_stride,
+                     float *err, int64_t err_stride, float lr, void *stream, int gt)
 {
     if (!c || !w || !grad) return A2SGD_ERR_ARG;
     if (!c->alg1 && !err) return A2SGD_ERR_ARG;
@@ -732,7 +749,7 @@ extern "C" int a2sgd_step_bf16(a2sgd_ctx *c, float *w, int64_t w_stride, const u
     {
         EncodeArgs a = make_encode_args(c, g, grad_stride, err, err_stride, c->local_means, c->pos_counts, nullptr,
                                         c->global_means);
-        const void *fn = select_encode_bf16(ef, vw_enc);
+        const void *fn = gt == 1 ? select_encode_lowp<1>(ef, vw_enc) : select_encode_lowp<2>(ef, vw_enc);
         const uint64_t items = vw_enc ? (c->n + 7) / 8 : c->n;
         const dim3 grid(std::min(per_worker_grid(c, occupancy(c, fn), items, A2SGD_WAVES_K1), c->g_alloc), c->P);
         void *params[] = {&a};
@@ -740,7 +757,8 @@ extern "C" int a2sgd_step_bf16(a2sgd_ctx *c, float *w, int64_t w_stride, const u
     }
     {
         DecodeArgs a = make_decode_args(c, w, ws, g, grad_stride, err, err_stride, c->local_means, c->global_means, lr);
-        const void *fn = select_decode_bf16(ef, store, ws == 0, c->P, vw_dec);
+        const void *fn = gt == 1 ? select_decode_lowp<1>(ef, store, ws == 0, c->P, vw_dec)
+                                 : select_decode_lowp<2>(ef, store, ws == 0, c->P, vw_dec);
         const uint64_t items = vw_dec ? (c->n + 7) / 8 : c->n;
         const dim3 grid = (ws == 0) ? dim3(flat_grid(c, occupancy(c, fn), items, A2SGD_WAVES_K3))
                                     : dim3(per_worker_grid(c, occupancy(c, fn), items, A2SGD_WAVES_K3), c->P);

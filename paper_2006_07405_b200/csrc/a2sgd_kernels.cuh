@@ -26,6 +26,7 @@
 // result depends only on (n, P, grid), never on scheduling.
 #pragma once
 
+#include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -122,10 +123,12 @@ __device__ __forceinline__ void st_stream1(float *p, float v)
     asm volatile("st.global.L1::no_allocate.f32 [%0], %1;" ::"l"(p), "f"(v) : "memory");
 }
 
-// A gradient row whose elements are fp32 (GB = false) or bfloat16 (GB = true; the paper notes that
-// the method "can be further integrated with quantization").  bfloat16 is the upper half of an
-// fp32, so widening is exact: v = float(g) + e is formed from exactly the value the caller stored.
-template <bool GB>
+// A gradient row whose elements are fp32 (GB = 0), bfloat16 (GB = 1) or IEEE half (GB = 2); the
+// paper notes that the method "can be further integrated with quantization".  Widening either
+// 16-bit format to fp32 is exact (bfloat16 is the upper half of an fp32; every half value,
+// subnormals included, is an fp32 value), so v = float(g) + e is formed from exactly the value the
+// caller stored.
+template <int GB>
 struct GradRow {
     const char *base;
     __device__ __forceinline__ GradRow(const float *grad_base, int64_t row_offset_elems)
@@ -137,7 +140,7 @@ struct GradRow {
         if (GB) {
             unsigned short h;
             asm volatile("ld.global.L1::no_allocate.u16 %0, [%1];" : "=h"(h) : "l"(base + 2 * elem));
-            return __uint_as_float((unsigned)h << 16);
+            return GB == 1 ? __uint_as_float((unsigned)h << 16) : __half2float(__ushort_as_half(h));
         }
         return ld_stream1(reinterpret_cast<const float *>(base) + elem);
     }
@@ -145,7 +148,7 @@ struct GradRow {
     __device__ __forceinline__ Vec<VW> vec(uint64_t elem) const
     {
         if (GB) {
-            static_assert(!GB || VW == 8, "bfloat16 gradients use 8-element (128-bit) vectors");
+            static_assert(!GB || VW == 8, "16-bit gradients use 8-element (128-bit) vectors");
             unsigned x[4];
             asm volatile("ld.global.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
                          : "=r"(x[0]), "=r"(x[1]), "=r"(x[2]), "=r"(x[3])
@@ -153,8 +156,13 @@ struct GradRow {
             Vec<VW> r;
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
-                r.v[2 * k] = __uint_as_float(x[k] << 16);
-                r.v[2 * k + 1] = __uint_as_float(x[k] & 0xffff0000u);
+                if (GB == 1) {
+                    r.v[2 * k] = __uint_as_float(x[k] << 16);
+                    r.v[2 * k + 1] = __uint_as_float(x[k] & 0xffff0000u);
+                } else {
+                    r.v[2 * k] = __half2float(__ushort_as_half((unsigned short)(x[k] & 0xffffu)));
+                    r.v[2 * k + 1] = __half2float(__ushort_as_half((unsigned short)(x[k] >> 16)));
+                }
             }
             return r;
         }
@@ -376,7 +384,7 @@ __device__ __forceinline__ void finish_worker(const EncodeArgs &a, uint32_t p, d
 // kernel would have done, so every value is bit-identical — and the new v is written back in
 // place.  The decode kernel then needs only the sign mask and w.  DEFER = 1: the buffer still
 // holds a true residual (first step, or after a2sgd_materialize_err); DEFER = 2: it holds v.
-template <bool EF, bool MASK, int VW, bool GB = false, int DEFER = 0>
+template <bool EF, bool MASK, int VW, int GB = 0, int DEFER = 0>
 __global__ void __launch_bounds__(kBlock) k_encode_vec(EncodeArgs a)
 {
     static_assert(DEFER == 0 || (EF && MASK && VW == 8 && !GB), "deferred residual: EF, mask, 256-bit, fp32 gradients");
@@ -499,7 +507,7 @@ __global__ void __launch_bounds__(kBlock) k_encode_vec(EncodeArgs a)
 }
 
 // General path: any 4-byte alignment, scalar coalesced accesses.  grid = (G, P).
-template <bool EF, bool MASK, bool GB = false>
+template <bool EF, bool MASK, int GB = 0>
 __global__ void __launch_bounds__(kBlock) k_encode_scalar(EncodeArgs a)
 {
     pdl_wait_prior_grid();
@@ -645,7 +653,7 @@ __device__ __forceinline__ Vec<VW> zero_vec()
 // workers in order (fixed summation order), so w is read and written once
 // per model element.  PT > 0: P known at compile time (all 2P+1 loads of a
 // vector are issued before any is used); PT == 0: run-time P.
-template <bool EF, bool STORE, int PT, int VW, bool GB = false>
+template <bool EF, bool STORE, int PT, int VW, int GB = 0>
 __global__ void __launch_bounds__(kBlock) k_decode_shared_vec(DecodeArgs a)
 {
     pdl_wait_prior_grid();
@@ -728,7 +736,7 @@ __global__ void __launch_bounds__(kBlock) k_decode_shared_vec(DecodeArgs a)
 }
 
 // One w replica per worker (Algorithm 1's layout).  grid = (G, P).
-template <bool EF, bool STORE, int VW, bool GB = false>
+template <bool EF, bool STORE, int VW, int GB = 0>
 __global__ void __launch_bounds__(kBlock) k_decode_repl_vec(DecodeArgs a)
 {
     pdl_wait_prior_grid();
@@ -788,7 +796,7 @@ __global__ void __launch_bounds__(kBlock) k_decode_repl_vec(DecodeArgs a)
 
 // General path: any 4-byte alignment, both weight layouts, scalar accesses.
 // Shared w: grid = (G, 1), the thread walks the workers; replicas: grid = (G, P).
-template <bool EF, bool STORE, bool GB = false>
+template <bool EF, bool STORE, int GB = 0>
 __global__ void __launch_bounds__(kBlock) k_decode_scalar(DecodeArgs a)
 {
     pdl_wait_prior_grid();

@@ -685,3 +685,33 @@ def test_pointer_check_flag_rejects_host_memory_before_any_launch():
     *_, status = B.a2sgd_read_stats(ctx)
     assert status == B.OK
     ctx.destroy()
+
+
+@pytest.mark.parametrize("mode", [EF, ALG1])
+@pytest.mark.parametrize("replicated", [False, True])
+@pytest.mark.parametrize("P,n,stride_pad,off", [(1, 9, 0, 0), (4, 1 << 20, 0, 0), (4, 100_003, 5, 0), (8, 33_333, 3, 1)])
+def test_f16_gradient_step_matches_oracle_on_widened_gradients(mode, replicated, P, n, stride_pad, off):
+    gen = torch.Generator("cuda").manual_seed(n + 3 * P)
+    stride = n + stride_pad
+    gbuf = torch.zeros(off + P * stride + 8, device="cuda")
+    gbuf.normal_(0.0, 1e-3, generator=gen)
+    gbuf[::7] *= 1e-4                                       # some values in the half-precision subnormal range
+    g16_all = gbuf.to(torch.float16)
+    g16 = g16_all[off:off + P * stride].view(P, stride)[:, :n]
+    # half -> fp32 by numpy's own conversion (exact): the oracle sees the widened values
+    gh = g16.contiguous().view(torch.int16).cpu().numpy().view(np.float16).astype(np.float32).reshape(P, n)
+    assert np.array_equal(gh, g16.float().cpu().numpy())
+    e = torch.empty((P, stride), device="cuda")[:, :n]
+    e.normal_(0.0, 3e-4, generator=gen)
+    w = (torch.empty((P, stride), device="cuda")[:, :n] if replicated else torch.empty(n, device="cuda"))
+    w.normal_(0.0, 0.02, generator=gen)
+    eh, wh = e.cpu().numpy().copy(), w.cpu().numpy().copy()
+    ctx = B.a2sgd_create(n, P, 0, mode)
+    B.a2sgd_step_f16(ctx, w, g16, e, 0.1)
+    lm, gm, cnt, status = B.a2sgd_read_stats(ctx)
+    lm_ref, gm_ref, cnt_ref = oracle.step(wh, gh, eh, 0.1, mode=mode)
+    assert status == B.OK and np.array_equal(cnt, cnt_ref)
+    assert_means(lm, lm_ref)
+    assert_means(gm, gm_ref)
+    assert_state(w.cpu().numpy(), wh, e.cpu().numpy(), eh, gm_ref, f"f16 P={P} n={n}")
+    ctx.destroy()
