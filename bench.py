@@ -15,6 +15,11 @@ workload.  Prints ONE JSON line (rank 0).
                  copy bandwidth of this machine.
 * ``cpu_baseline`` the CPU oracle, as it stands, on a bounded sample of the same workload.
 
+The default workload at N = 1 is the largest benchmark configuration, c5_gpt2_xl (1.56 G
+parameters, P = 4, 56 GB resident); if the device cannot hold it the run falls back to c4_vgg16
+and says so in ``config``.  The smaller configurations are timed too and reported under
+``other_workloads`` with their own per-kernel roofline records.
+
 With N > 1 (under torchrun) every rank runs an independent replica of the workload on its own
 GPU — the benchmarked path has no exchange between GPUs — and the time is the max over ranks.
 """
@@ -41,6 +46,8 @@ FALLBACK_HBM_GBS = 6650.0
 # captures summarised under profiles/ (None until a capture exists for that P).
 NCU_DECODE_TRAFFIC_PER_ELEMENT = {4: 52.92}  # 36.0 read + 16.92 written inside the launch; 3.08 B/element of
 #                                               dirty lines leave L2 during the next launch
+DEFAULT_WORKLOAD = "c5_gpt2_xl"
+FALLBACK_WORKLOAD = "c4_vgg16"
 
 
 def algorithmic_bytes_per_model_element(P: int, shared_w: bool = True) -> dict:
@@ -248,7 +255,35 @@ def whole_job_value(n_model: int, n_replicas: int, ms_per_step: float) -> float:
     return n_replicas * n_model / (ms_per_step * 1e-3)
 
 
-def time_workload(wl, steps, warmup, dev, *, with_roofline=True, with_e2e=True, dist=None):
+def spread(samples) -> dict:
+    """median / min / max of a list of per-step (or per-launch) milliseconds."""
+    xs = sorted(float(x) for x in samples)
+    if not xs:
+        return {"n": 0}
+    mid = len(xs) // 2
+    med = xs[mid] if len(xs) % 2 else 0.5 * (xs[mid - 1] + xs[mid])
+    return {"median": med, "min": xs[0], "max": xs[-1], "n": len(xs)}
+
+
+def host_description() -> dict:
+    """Core count and CPU model of the box the oracle is timed on."""
+    model = None
+    try:
+        with open("/proc/cpuinfo") as f:
+            for line in f:
+                if line.lower().startswith("model name"):
+                    model = line.split(":", 1)[1].strip()
+                    break
+    except OSError:
+        pass
+    try:
+        usable = len(os.sched_getaffinity(0))
+    except AttributeError:
+        usable = os.cpu_count()
+    return {"nproc": os.cpu_count(), "usable_cores": usable, "cpu_model": model}
+
+
+def time_workload(wl, steps, warmup, dev, *, with_roofline=True, with_next_rows=True, with_e2e=True, dist=None):
     """Runs the timed regions for one workload on this rank's GPU.  Returns a dict of results."""
     import torch
     from paper_2006_07405_b200 import binding as B
@@ -294,20 +329,23 @@ def time_workload(wl, steps, warmup, dev, *, with_roofline=True, with_e2e=True, 
             graph, chunk = None, 1
             sys.stderr.write(f"CUDA graph capture failed ({ex}); timing eager launches\n")
         barrier()
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    # One event before every step (or graph replay) and one after the last: the K steps are timed
+    # as one region (first to last event); the events in between give the spread.
+    marks = [torch.cuda.Event(enable_timing=True) for _ in range(steps // chunk + 1)]
     wall0 = time.time()
-    ev0.record()
-    if graph is not None:
-        for _ in range(steps // chunk):
+    for i in range(steps // chunk):
+        marks[i].record()
+        if graph is not None:
             graph.replay()
-    else:
-        for _ in range(steps):
+        else:
             B.a2sgd_step(ctx, w, g, e, wl.lr)
-    ev1.record()
+    marks[-1].record()
     barrier()
     wall1 = time.time()
-    ms = max_over_ranks(ev0.elapsed_time(ev1), dist, dev)
+    ms = max_over_ranks(marks[0].elapsed_time(marks[-1]), dist, dev)
+    per_step = [marks[i].elapsed_time(marks[i + 1]) / chunk for i in range(len(marks) - 1)]
     res = {"ms_total": ms, "ms_per_step": ms / steps, "launches": launches_per_step * steps,
+           "step_ms_spread": spread(per_step),
            "launch_info": info, "wall": (wall0, wall1),
            "launch_mode": f"CUDA graph of {chunk} steps" if graph is not None else "eager"}
     del graph
@@ -315,11 +353,10 @@ def time_workload(wl, steps, warmup, dev, *, with_roofline=True, with_e2e=True, 
     res["device_status"] = status
 
     if with_roofline:
-        # the decode/update kernel alone, same launch configuration as inside a2sgd_step
+        # the two kernels of a step each timed alone, in the launch configuration a2sgd_step uses
         lm = torch.zeros((P, 2), device=dev)
         gm = torch.zeros(2, device=dev)
         k_steps = max(5, min(steps, 200))
-        enc_ms = dec_ms = 0.0
         evs = [torch.cuda.Event(enable_timing=True) for _ in range(3 * k_steps)]
         for i in range(k_steps):
             evs[3 * i].record()
@@ -329,48 +366,41 @@ def time_workload(wl, steps, warmup, dev, *, with_roofline=True, with_e2e=True, 
             B.a2sgd_decode_update(ctx, w, g, e, lm, gm, wl.lr)
             evs[3 * i + 2].record()
         torch.cuda.synchronize(dev)
-        for i in range(k_steps):
-            enc_ms += evs[3 * i].elapsed_time(evs[3 * i + 1])
-            dec_ms += evs[3 * i + 1].elapsed_time(evs[3 * i + 2])
-        res["encode_ms"] = enc_ms / k_steps
-        res["decode_ms"] = dec_ms / k_steps
+        enc = [evs[3 * i].elapsed_time(evs[3 * i + 1]) for i in range(k_steps)]
+        dec = [evs[3 * i + 1].elapsed_time(evs[3 * i + 2]) for i in range(k_steps)]
+        res["encode_ms"] = sum(enc) / k_steps
+        res["decode_ms"] = sum(dec) / k_steps
+        res["encode_ms_spread"] = spread(enc)
+        res["decode_ms_spread"] = spread(dec)
 
-    if with_roofline:
-        # rows beyond the core step: the dense synchronisation step (Algorithm 1 lines 9-10) and the
-        # same step over a segment list (one tensor per segment of the workload)
+    if with_next_rows:
+        # rows beyond the core step: the dense synchronisation step (Algorithm 1 lines 9-10), the
+        # deferred-residual and 16-bit-gradient forms, and the step over a segment list
         k_steps = max(5, min(steps, 50))
         evs = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
-        for _ in range(3):
-            B.a2sgd_dense_sync(ctx, w, g, wl.lr)
-        evs[0].record()
-        for _ in range(k_steps):
-            B.a2sgd_dense_sync(ctx, w, g, wl.lr)
-        evs[1].record()
-        torch.cuda.synchronize(dev)
-        res["dense_sync_ms"] = evs[0].elapsed_time(evs[1]) / k_steps
-        if g.stride(0) % 8 == 0:
-            dctx = B.a2sgd_create(n, P, dev.index, B.MODE_EF | B.DEFERRED_RESIDUAL)
+
+        def timed(call):
             for _ in range(3):
-                B.a2sgd_step(dctx, w, g, e, wl.lr)
+                call()
             evs[0].record()
             for _ in range(k_steps):
-                B.a2sgd_step(dctx, w, g, e, wl.lr)
+                call()
             evs[1].record()
+            torch.cuda.synchronize(dev)
+            return evs[0].elapsed_time(evs[1]) / k_steps
+
+        res["dense_sync_ms"] = timed(lambda: B.a2sgd_dense_sync(ctx, w, g, wl.lr))
+        if g.stride(0) % 8 == 0:
+            dctx = B.a2sgd_create(n, P, dev.index, B.MODE_EF | B.DEFERRED_RESIDUAL)
+            res["step_deferred_ms"] = timed(lambda: B.a2sgd_step(dctx, w, g, e, wl.lr))
             B.a2sgd_materialize_err(dctx, e)
             torch.cuda.synchronize(dev)
-            res["step_deferred_ms"] = evs[0].elapsed_time(evs[1]) / k_steps
             dctx.destroy()
         g16 = torch.empty((P, g.stride(0)), dtype=torch.bfloat16, device=dev)[:, :n]
         g16.copy_(g)
-        for _ in range(3):
-            B.a2sgd_step_bf16(ctx, w, g16, e, wl.lr)
-        evs[0].record()
-        for _ in range(k_steps):
-            B.a2sgd_step_bf16(ctx, w, g16, e, wl.lr)
-        evs[1].record()
-        torch.cuda.synchronize(dev)
-        res["step_bf16_ms"] = evs[0].elapsed_time(evs[1]) / k_steps
+        res["step_bf16_ms"] = timed(lambda: B.a2sgd_step_bf16(ctx, w, g16, e, wl.lr))
         del g16
+        torch.cuda.empty_cache()
         free_b, _ = torch.cuda.mem_get_info(dev)
         if hasattr(wl, "segments") and free_b > (2 * P + 1) * n * 4 * 1.1:
             sizes = [sg.numel for sg in wl.segments]
@@ -378,37 +408,35 @@ def time_workload(wl, steps, warmup, dev, *, with_roofline=True, with_e2e=True, 
             es = [[t.clone() for t in torch.split(e[p], sizes)] for p in range(P)]
             ws = [t.clone() for t in torch.split(w, sizes)]
             plan = B.a2sgd_segments_create(ctx, gs, es, ws)
-            for _ in range(3):
-                B.a2sgd_step_segments(ctx, plan, wl.lr)
-            evs[0].record()
-            for _ in range(k_steps):
-                B.a2sgd_step_segments(ctx, plan, wl.lr)
-            evs[1].record()
-            torch.cuda.synchronize(dev)
-            res["step_segments_ms"] = evs[0].elapsed_time(evs[1]) / k_steps
+            res["step_segments_ms"] = timed(lambda: B.a2sgd_step_segments(ctx, plan, wl.lr))
             plan.destroy()
             del gs, es, ws, plan
             torch.cuda.empty_cache()
 
     if with_e2e:
+        pinned = True
         try:
-            g_host = torch.empty((P, n)).pin_memory()
-        except Exception:
-            g_host = torch.empty((P, n))
+            g_host = torch.empty((P, n), pin_memory=True)
+        except Exception as ex:
+            sys.stderr.write(f"pinned allocation of {P * n * 4 / 1e9:.1f} GB failed ({ex}); pageable host memory\n")
+            g_host, pinned = torch.empty((P, n)), False
         g_host.copy_(g)
         means = torch.zeros(2 * P + 2).pin_memory()
-        e2e_steps = max(2, min(steps, 10))
+        e2e_steps = max(2, min(steps, 10 if n * P < (1 << 30) else 3))
         for _ in range(2):
             B.a2sgd_step_host(ctx, w, g_host, g, e, wl.lr, means)
         barrier()
-        ev0.record()
-        for _ in range(e2e_steps):
+        marks = [torch.cuda.Event(enable_timing=True) for _ in range(e2e_steps + 1)]
+        for i in range(e2e_steps):
+            marks[i].record()
             B.a2sgd_step_host(ctx, w, g_host, g, e, wl.lr, means)
-        ev1.record()
+        marks[-1].record()
         barrier()
-        ms2 = max_over_ranks(ev0.elapsed_time(ev1), dist, dev)
+        ms2 = max_over_ranks(marks[0].elapsed_time(marks[-1]), dist, dev)
         res["e2e_ms_per_step"] = ms2 / e2e_steps
+        res["e2e_ms_spread"] = spread([marks[i].elapsed_time(marks[i + 1]) for i in range(e2e_steps)])
         res["e2e_steps"] = e2e_steps
+        res["e2e_pinned"] = pinned
         res["h2d_bytes"] = P * n * 4
         res["d2h_bytes"] = (2 * P + 2) * 4
         del g_host
@@ -429,39 +457,104 @@ def load_loop_for_clocks(wl, dev, seconds):
     w = torch.zeros(n, device=dev)
     W.fill_gradients(wl, 0, g)
     ctx = B.a2sgd_create(n, P, dev.index, B.MODE_EF)
+    per_sync = 50 if n * P < (1 << 30) else 5
     t0 = time.time()
     while time.time() - t0 < seconds:
-        for _ in range(50):
+        for _ in range(per_sync):
             B.a2sgd_step(ctx, w, g, e, wl.lr)
         torch.cuda.synchronize(dev)
     ctx.destroy()
 
 
+def kernel_rooflines(wl, res, peak_gbs) -> dict:
+    """Per-kernel roofline records (K1 encode-reduce, K3 decode/update) from the per-launch event
+    times of ``time_workload``: algorithmic bytes / launch duration against the measured peak."""
+    b = algorithmic_bytes_per_model_element(wl.P)
+    out = {}
+    for key, name in (("encode", "encode-reduce (K1) + stand-alone global-average launch"),
+                      ("decode", "decode/update (K3)")):
+        ms = res[f"{key}_ms"]
+        achieved = b[key] * wl.n / (ms * 1e-3) / 1e9
+        out[key] = {"bound": "hbm", "kernel": name, "achieved": achieved, "peak": peak_gbs, "unit": "GB/s",
+                    "frac": achieved / peak_gbs, "frac_of_8TBps": achieved / NOMINAL_HBM_GBS,
+                    "algorithmic_bytes": b[key] * wl.n, "launch_ms": ms, "launch_ms_spread": res[f"{key}_ms_spread"]}
+    return out
+
+
 def summarise(wl, res, n_gpus, peak_gbs):
     b = algorithmic_bytes_per_model_element(wl.P)
     t = res["ms_per_step"] * 1e-3
-    out = {"n": wl.n, "P": wl.P, "ms_per_step": res["ms_per_step"], "launch_mode": res["launch_mode"],
+    out = {"n": wl.n, "P": wl.P, "ms_per_step": res["ms_per_step"], "step_ms_spread": res["step_ms_spread"],
+           "launch_mode": res["launch_mode"],
            "single_launch": res["launch_info"]["single_launch"],
            "model_params_per_s": n_gpus * wl.n / t, "worker_params_per_s": n_gpus * wl.n * wl.P / t,
            "step_GBps": b["step"] * wl.n / t / 1e9,
            "step_frac_of_8TBps": b["step"] * wl.n / t / 1e9 / NOMINAL_HBM_GBS,
            "step_frac_of_measured_peak": b["step"] * wl.n / t / 1e9 / peak_gbs}
     if "decode_ms" in res:
-        out["encode_ms"] = res["encode_ms"]
-        out["decode_ms"] = res["decode_ms"]
-        out["encode_GBps"] = b["encode"] * wl.n / (res["encode_ms"] * 1e-3) / 1e9
-        out["decode_GBps"] = b["decode"] * wl.n / (res["decode_ms"] * 1e-3) / 1e9
+        out["roofline"] = kernel_rooflines(wl, res, peak_gbs)
+    rows = next_rows_of(wl, res, peak_gbs)
+    if rows:
+        out["next_rows"] = rows
     return out
+
+
+def next_rows_of(wl, res, peak_gbs) -> dict:
+    b = algorithmic_bytes_per_model_element(wl.P)
+    rows = {}
+    if "dense_sync_ms" in res:
+        bts = (4 * wl.P + 8) * wl.n
+        rows["dense_sync (Algorithm 1 lines 9-10)"] = {
+            "ms": res["dense_sync_ms"], "GBps": bts / (res["dense_sync_ms"] * 1e-3) / 1e9,
+            "frac_of_measured_peak": bts / (res["dense_sync_ms"] * 1e-3) / 1e9 / peak_gbs,
+            "bytes_per_model_element": 4 * wl.P + 8}
+    if "step_segments_ms" in res:
+        bts = b["step"] * wl.n
+        rows["step over a segment list (one tensor per segment)"] = {
+            "ms": res["step_segments_ms"], "GBps": bts / (res["step_segments_ms"] * 1e-3) / 1e9,
+            "frac_of_8TBps": bts / (res["step_segments_ms"] * 1e-3) / 1e9 / NOMINAL_HBM_GBS,
+            "segments": len(wl.segments)}
+    if "step_deferred_ms" in res:
+        bts = (12 * wl.P + 8 + wl.P / 4) * wl.n
+        rows["step, deferred-residual representation (opt-in, bit-identical results)"] = {
+            "ms": res["step_deferred_ms"], "GBps_actual_bytes": bts / (res["step_deferred_ms"] * 1e-3) / 1e9,
+            "model_params_per_s": wl.n / (res["step_deferred_ms"] * 1e-3),
+            "bytes_per_model_element": 12 * wl.P + 8 + wl.P / 4,
+            "speedup_vs_canonical_step": res["ms_per_step"] / res["step_deferred_ms"]}
+    if "step_bf16_ms" in res:
+        bts = (16 * wl.P + 8) * wl.n
+        rows["step with bfloat16 gradients"] = {
+            "ms": res["step_bf16_ms"], "GBps": bts / (res["step_bf16_ms"] * 1e-3) / 1e9,
+            "frac_of_8TBps": bts / (res["step_bf16_ms"] * 1e-3) / 1e9 / NOMINAL_HBM_GBS,
+            "model_params_per_s": wl.n / (res["step_bf16_ms"] * 1e-3), "bytes_per_model_element": 16 * wl.P + 8}
+    return rows
+
+
+def pick_workload(name, scale_div, dev):
+    """The requested workload, or the fallback when the device cannot hold its resident set."""
+    import torch
+    from paper_2006_07405_b200 import workloads as W
+    wl = W.get_workload(name)
+    if scale_div > 1:
+        wl = W.scaled(wl, scale_div)
+    note = None
+    free_b, _ = torch.cuda.mem_get_info(dev)
+    need = (2 * wl.P + 1) * wl.n * 4 * 1.05
+    if need > free_b and name == DEFAULT_WORKLOAD and scale_div == 1:
+        note = (f"{name} needs {need / 1e9:.0f} GB of device memory, {free_b / 1e9:.0f} GB free: "
+                f"fell back to {FALLBACK_WORKLOAD}")
+        wl = W.get_workload(FALLBACK_WORKLOAD)
+    return wl, note
 
 
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--steps", type=int, default=60)
     ap.add_argument("--warmup", type=int, default=5)
-    ap.add_argument("--workload", default="c2_lstm_ptb")
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
     ap.add_argument("--impl", default="native", choices=["native", "reference"])
-    ap.add_argument("--no-extra", action="store_true", help="skip the extra c4/c5 measurements at N=1")
+    ap.add_argument("--no-extra", action="store_true", help="skip the other configurations at N=1")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--scale-div", type=int, default=1,
                     help="divide every tensor length of the workload (small cases for profiler captures)")
@@ -499,9 +592,7 @@ def main():
     n_gpus = world
     dev = torch.device("cuda", local_rank)
     torch.cuda.set_device(dev)
-    wl = W.get_workload(args.workload)
-    if args.scale_div > 1:
-        wl = W.scaled(wl, args.scale_div)
+    wl, fallback_note = pick_workload(args.workload, args.scale_div, dev)
     peak_gbs, peak_src = measured_peak_gbs()
     steps, warmup = max(1, args.steps), max(3, args.warmup)
 
@@ -511,7 +602,8 @@ def main():
                           "note": "minimal run for profiler captures"}), flush=True)
         return
     if args.minimal:
-        res = time_workload(wl, steps, warmup, dev, with_roofline=False, with_e2e=False, dist=dist)
+        res = time_workload(wl, steps, warmup, dev, with_roofline=False, with_next_rows=False, with_e2e=False,
+                            dist=dist)
         if rank == 0:
             print(json.dumps({"metric": METRIC, "value": n_gpus * wl.n / (res["ms_per_step"] * 1e-3), "unit": UNIT,
                               "ms_per_step": res["ms_per_step"], "steps": steps, "warmup": warmup,
@@ -529,12 +621,13 @@ def main():
             "timed region plus 1.5 s of the same step loop (timed region shorter than the sampling period allows)"
 
     extra = {}
-    if rank == 0 and world == 1 and not args.no_extra and args.workload == "c2_lstm_ptb" and args.scale_div == 1:
-        free_b, _ = torch.cuda.mem_get_info(dev)
-        for name in ("c1_flat_1m", "c3_resnet50", "c4_vgg16", "c5_gpt2_xl"):
+    if rank == 0 and world == 1 and not args.no_extra and args.scale_div == 1:
+        for name in ("c1_flat_1m", "c2_lstm_ptb", "c3_resnet50", "c4_vgg16", "c5_gpt2_xl"):
+            if name == wl.name:
+                continue
             w2 = W.get_workload(name)
-            need = (2 * w2.P + 1) * w2.n * 4 * 1.05
-            if need > free_b:
+            free_b, _ = torch.cuda.mem_get_info(dev)
+            if (2 * w2.P + 1) * w2.n * 4 * 1.05 > free_b:
                 extra[name] = {"skipped": "not enough free device memory"}
                 continue
             k = 20 if w2.n > 10 ** 9 else (100 if w2.n > 10 ** 7 else 1000)
@@ -551,72 +644,48 @@ def main():
     b = algorithmic_bytes_per_model_element(wl.P)
     t = res["ms_per_step"] * 1e-3
     value = whole_job_value(wl.n, n_gpus, res["ms_per_step"])
-    dec_t = res["decode_ms"] * 1e-3
-    achieved = b["decode"] * wl.n / dec_t / 1e9
+    roofs = kernel_rooflines(wl, res, peak_gbs)
     traffic_per_el = NCU_DECODE_TRAFFIC_PER_ELEMENT.get(wl.P)
+    config = dict(W.describe(wl), mode="EF", w_layout="one shared w", resident_GB=(2 * wl.P + 1) * wl.n * 4 / 1e9,
+                  l2="inputs larger than L2: every step streams the whole resident set",
+                  parallelism=f"{n_gpus} independent replica(s), no collective",
+                  worker_params_per_s=n_gpus * wl.n * wl.P / t,
+                  step_GBps=b["step"] * wl.n / t / 1e9,
+                  step_frac_of_8TBps=b["step"] * wl.n / t / 1e9 / NOMINAL_HBM_GBS,
+                  step_frac_of_measured_peak=b["step"] * wl.n / t / 1e9 / peak_gbs,
+                  step_ms_spread=res["step_ms_spread"],
+                  bytes_per_model_element=b, launch=res["launch_info"], launch_mode=res["launch_mode"],
+                  row_stride="n rounded up to 32 elements (rows start 128-byte aligned)",
+                  encode_ms=res["encode_ms"], decode_ms=res["decode_ms"],
+                  device_status=res["device_status"])
+    if fallback_note:
+        config["fallback"] = fallback_note
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": n_gpus, "steps": steps, "warmup": warmup,
         "ms_per_step": res["ms_per_step"], "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f32", "data": "synthetic",
-        "config": dict(W.describe(wl), mode="EF", w_layout="one shared w", resident_GB=(2 * wl.P + 1) * wl.n * 4 / 1e9,
-                       l2="inputs larger than L2: every step streams the whole resident set",
-                       parallelism=f"{n_gpus} independent replica(s), no collective",
-                       worker_params_per_s=n_gpus * wl.n * wl.P / t,
-                       step_GBps=b["step"] * wl.n / t / 1e9,
-                       step_frac_of_8TBps=b["step"] * wl.n / t / 1e9 / NOMINAL_HBM_GBS,
-                       step_frac_of_measured_peak=b["step"] * wl.n / t / 1e9 / peak_gbs,
-                       bytes_per_model_element=b, launch=res["launch_info"], launch_mode=res["launch_mode"],
-                       row_stride="n rounded up to 32 elements (rows start 128-byte aligned)",
-                       encode_ms=res["encode_ms"], decode_ms=res["decode_ms"],
-                       device_status=res["device_status"]),
+        "config": config,
         "gpu_launches": res["launches"],
         "clocks": clocks,
         "e2e": {"value": n_gpus * wl.n / (res["e2e_ms_per_step"] * 1e-3), "unit": UNIT,
                 "h2d_bytes_per_step": res["h2d_bytes"], "d2h_bytes_per_step": res["d2h_bytes"],
-                "ms_per_step": res["e2e_ms_per_step"], "steps": res["e2e_steps"],
+                "ms_per_step": res["e2e_ms_per_step"], "ms_spread": res["e2e_ms_spread"], "steps": res["e2e_steps"],
+                "host_memory": "pinned" if res["e2e_pinned"] else "pageable (pinned allocation failed)",
                 "api": "a2sgd_step_host (pinned host gradients in, 2P+2 means out)"},
-        "roofline": {"bound": "hbm", "kernel": "decode/update (K3)", "achieved": achieved, "peak": peak_gbs,
-                     "unit": "GB/s", "frac": achieved / peak_gbs, "peak_source": peak_src,
-                     "traffic": traffic_per_el * wl.n if traffic_per_el else None,
-                     "algorithmic_bytes": b["decode"] * wl.n, "launch_ms": res["decode_ms"],
-                     "encode_kernel": {"achieved": b["encode"] * wl.n / (res["encode_ms"] * 1e-3) / 1e9,
-                                       "frac": b["encode"] * wl.n / (res["encode_ms"] * 1e-3) / 1e9 / peak_gbs,
-                                       "launch_ms": res["encode_ms"],
-                                       "note": "encode + stand-alone global-average launch"}},
+        "roofline": dict(roofs["decode"], peak_source=peak_src,
+                         traffic=traffic_per_el * wl.n if traffic_per_el else None,
+                         traffic_source="ncu dram__bytes read+write per model element of a smaller capture of the "
+                                        "same kernel (profiles/), scaled by n" if traffic_per_el else None,
+                         encode_kernel=roofs["encode"]),
     }
-    next_rows = {}
-    if "dense_sync_ms" in res:
-        bts = (4 * wl.P + 8) * wl.n
-        next_rows["dense_sync (Algorithm 1 lines 9-10)"] = {
-            "ms": res["dense_sync_ms"], "GBps": bts / (res["dense_sync_ms"] * 1e-3) / 1e9,
-            "frac_of_measured_peak": bts / (res["dense_sync_ms"] * 1e-3) / 1e9 / peak_gbs,
-            "bytes_per_model_element": 4 * wl.P + 8}
-    if "step_segments_ms" in res:
-        bts = b["step"] * wl.n
-        next_rows["step over a segment list (one tensor per segment)"] = {
-            "ms": res["step_segments_ms"], "GBps": bts / (res["step_segments_ms"] * 1e-3) / 1e9,
-            "frac_of_8TBps": bts / (res["step_segments_ms"] * 1e-3) / 1e9 / NOMINAL_HBM_GBS,
-            "segments": len(wl.segments)}
-    if "step_deferred_ms" in res:
-        bts = (12 * wl.P + 8 + wl.P / 4) * wl.n
-        next_rows["step, deferred-residual representation (opt-in, bit-identical results)"] = {
-            "ms": res["step_deferred_ms"], "GBps_actual_bytes": bts / (res["step_deferred_ms"] * 1e-3) / 1e9,
-            "model_params_per_s": wl.n / (res["step_deferred_ms"] * 1e-3),
-            "bytes_per_model_element": 12 * wl.P + 8 + wl.P / 4,
-            "speedup_vs_canonical_step": res["ms_per_step"] / res["step_deferred_ms"]}
-    if "step_bf16_ms" in res:
-        bts = (16 * wl.P + 8) * wl.n
-        next_rows["step with bfloat16 gradients"] = {
-            "ms": res["step_bf16_ms"], "GBps": bts / (res["step_bf16_ms"] * 1e-3) / 1e9,
-            "frac_of_8TBps": bts / (res["step_bf16_ms"] * 1e-3) / 1e9 / NOMINAL_HBM_GBS,
-            "model_params_per_s": wl.n / (res["step_bf16_ms"] * 1e-3), "bytes_per_model_element": 16 * wl.P + 8}
-    if next_rows:
-        line["next_rows"] = next_rows
+    rows = next_rows_of(wl, res, peak_gbs)
+    if rows:
+        line["next_rows"] = rows
     if extra:
         line["other_workloads"] = extra
     if not args.no_cpu_baseline and world == 1:
         cb = oracle_sample_rate(wl, 10.0)
-        line["cpu_baseline"] = {k: v for k, v in cb.items() if not k.startswith("_")}
+        line["cpu_baseline"] = dict({k: v for k, v in cb.items() if not k.startswith("_")}, host=host_description())
     print(json.dumps(line), flush=True)
     if dist is not None:
         dist.destroy_process_group()

@@ -1103,10 +1103,20 @@ __device__ __forceinline__ bool coop_reduce_and_barrier(const CoopArgs &a, Acc (
         sh.generation = ld_acquire_u32(&a.barrier[1]);
         __threadfence();
         const unsigned int t = atomicAdd(&a.barrier[0], 1u);
-        sh.flag = (t == a.expected - 1) ? 1 : 0;
+        int role = (t == a.expected - 1) ? 1 : 0;
+        // A CTA that gave up has written nothing.  If one already did, the last arriver leaves the
+        // barrier shut, so the remaining CTAs run out too and the step is abandoned as a whole
+        // (best effort: a CTA may still give up just after this check).
+        if (role == 1 && ld_acquire_u32(reinterpret_cast<const unsigned int *>(ea.status)) == (unsigned int)kDevTimeout)
+            role = -1;
+        sh.flag = role;
     }
     __syncthreads();
-    if (sh.flag) {
+    // every thread takes its own copy before the word is reused for the outcome of the wait below
+    const int role = sh.flag;
+    __syncthreads();
+    if (role < 0) return false;
+    if (role == 1) {
         __threadfence();
         // kWarps / PT warps fold each worker's G partials: thread tg of the group takes partials
         // tg, tg + group size, ... (index order), then a fixed tree inside the group
