@@ -61,6 +61,10 @@ def _load():
             ctypes.c_int, ctypes.c_uint64, ctypes.c_uint32, f32p, ctypes.c_int64,
             f32p, ctypes.c_int64, f32p, ctypes.c_int64, ctypes.c_float,
             f32p, f32p, u64p]
+        lib.a2sgd_oracle_decode_update_momentum.restype = ctypes.c_int
+        lib.a2sgd_oracle_decode_update_momentum.argtypes = [
+            ctypes.c_int, ctypes.c_uint64, ctypes.c_uint32, f32p, ctypes.c_int64, f32p, ctypes.c_int64,
+            f32p, ctypes.c_int64, f32p, ctypes.c_int64, f32p, f32p, ctypes.c_float, ctypes.c_float, ctypes.c_float]
         lib.a2sgd_oracle_dense_sync.restype = ctypes.c_int
         lib.a2sgd_oracle_dense_sync.argtypes = [
             ctypes.c_uint64, ctypes.c_uint32, f32p, ctypes.c_int64, f32p, ctypes.c_int64, ctypes.c_float]
@@ -134,6 +138,34 @@ def decode_update(w, grad, err, local_means, global_means, lr, *, mode=MODE_EF, 
         mode, n, P, wp, ws, gp, gs, ep, es,
         lm.ctypes.data_as(ctypes.POINTER(ctypes.c_float)) if lm is not None else None,
         gm.ctypes.data_as(ctypes.POINTER(ctypes.c_float)), lr), "decode_update")
+
+
+def decode_update_momentum(w, mom, grad, err, local_means, global_means, lr, beta, weight_decay, *,
+                           mode=MODE_EF, n=None):
+    """Decode / residual / update with heavy-ball momentum and weight decay, in place:
+    m <- beta*m + g_hat + weight_decay*w;  w <- w - lr*m.  ``mom`` has the layout of ``w``."""
+    lib = _load()
+    P = grad.shape[0]
+    n = grad.shape[1] if n is None else n
+    gp, gs = _rows(grad, "grad")
+    ep, es = _rows(err, "err") if err is not None else (None, 0)
+    wp, ws = _weights(w, P)
+    mp, ms = _weights(mom, P)
+    lm = np.ascontiguousarray(local_means, np.float32) if local_means is not None else None
+    gm = np.ascontiguousarray(global_means, np.float32)
+    _check(lib.a2sgd_oracle_decode_update_momentum(
+        mode, n, P, wp, ws, mp, ms, gp, gs, ep, es,
+        lm.ctypes.data_as(ctypes.POINTER(ctypes.c_float)) if lm is not None else None,
+        gm.ctypes.data_as(ctypes.POINTER(ctypes.c_float)), lr, beta, weight_decay), "decode_update_momentum")
+
+
+def step_momentum(w, mom, grad, err, lr, beta, weight_decay, *, mode=MODE_EF, n=None):
+    """encode -> global_average -> decode_update_momentum, the three oracle calls in order.
+    Returns (local_means, global_means, pos_counts)."""
+    lm, cnt, _ = encode(grad, err if mode == MODE_EF else None, mode=mode, n=n)
+    gm = global_average(lm)
+    decode_update_momentum(w, mom, grad, err, lm, gm, lr, beta, weight_decay, mode=mode, n=n)
+    return lm, gm, cnt
 
 
 def step(w, grad, err, lr, *, mode=MODE_EF, n=None):

@@ -424,3 +424,120 @@ def test_dense_sync_after_identical_local_steps_equals_eq1():
     w = np.array([10, 10, 10], np.float32)
     oracle.dense_sync(w, g, 0.5)
     assert w.tolist() == [9.0, 10.0, 11.0]
+
+
+# ---------------------------------------------------------------- momentum / weight decay on the reconstructed gradient
+def test_golden_m1_momentum_and_weight_decay_two_steps():
+    fx = _load("m1_momentum_weight_decay_two_steps.json")
+    for case in fx["cases"]:
+        w = np.array(fx["w0"], np.float32)
+        m = np.array(fx["m0"], np.float32)
+        e = _f32(fx["e0"])
+        for t in range(2):
+            g = _f32(fx["g"][t])
+            oracle.step_momentum(w, m, g, e, fx["lr"], case["beta"], case["weight_decay"], mode=EF)
+            assert e.tolist() == fx["e"][t]
+            assert m.tolist() == case["m"][t]
+            assert w.tolist() == case["w"][t]
+
+
+@pytest.mark.parametrize("mode", [EF, ALG1])
+@pytest.mark.parametrize("replicated", [False, True])
+def test_momentum_with_beta_zero_and_no_decay_is_the_plain_step_bit_for_bit(mode, replicated):
+    rng = np.random.default_rng(11)
+    P, n = 3, 257
+    g = (rng.standard_normal((P, n)) * 1e-2).astype(np.float32)
+    e0 = (rng.standard_normal((P, n)) * 3e-3).astype(np.float32)
+    w0 = (rng.standard_normal((P, n) if replicated else n) * 0.02).astype(np.float32)
+    lm, cnt, _ = oracle.encode(g, e0 if mode == EF else None, mode=mode)
+    gm = oracle.global_average(lm)
+    w_a, e_a = w0.copy(), e0.copy()
+    oracle.decode_update(w_a, g, e_a, lm, gm, 0.1, mode=mode)
+    w_b, e_b = w0.copy(), e0.copy()
+    m = (rng.standard_normal(w0.shape)).astype(np.float32)       # beta = 0: the old buffer must not matter
+    oracle.decode_update_momentum(w_b, m, g, e_b, lm, gm, 0.1, 0.0, 0.0, mode=mode)
+    assert np.array_equal(w_a, w_b) and np.array_equal(e_a, e_b)
+    # and the buffer now holds g_hat itself: w0 - lr*m reproduces w up to the two roundings
+    assert np.allclose(w0.astype(np.float64) - np.float32(0.1).astype(np.float64) * m, w_b, rtol=0, atol=1e-8)
+
+
+def test_momentum_constant_gradient_closed_form():
+    """A two-valued gradient with e = 0 and one worker is reconstructed exactly (g_hat = g, no
+    residual), so every step feeds the same g_hat: m_t = g_hat (1 - beta^t) / (1 - beta) and
+    w_t = w_0 - lr * sum_{s<=t} m_s."""
+    n, beta, lr, T = 64, 0.5, 0.25, 6
+    g = np.where(np.arange(n) % 3 == 0, 0.75, -0.5).astype(np.float32)[None, :]
+    w = np.linspace(-1, 1, n).astype(np.float32)
+    w0 = w.astype(np.float64).copy()
+    m = np.zeros(n, np.float32)
+    e = np.zeros((1, n), np.float32)
+    acc = np.zeros(n)
+    for t in range(1, T + 1):
+        oracle.step_momentum(w, m, g, e, lr, beta, 0.0, mode=EF)
+        assert not e.any()
+        m_exact = g[0].astype(np.float64) * (1 - beta ** t) / (1 - beta)
+        acc += m_exact
+        assert np.allclose(m, m_exact, rtol=1e-7, atol=0)
+        assert np.allclose(w, w0 - lr * acc, rtol=0, atol=2e-7)
+
+
+def test_weight_decay_alone_shrinks_the_weights():
+    """beta = 0: w <- w (1 - lr*wd) - lr*g_hat."""
+    rng = np.random.default_rng(5)
+    P, n, lr, wd = 2, 100, 0.5, 0.125
+    g = rng.standard_normal((P, n)).astype(np.float32)
+    e = np.zeros((P, n), np.float32)
+    w0 = rng.standard_normal(n).astype(np.float32)
+    w_plain, e1 = w0.copy(), e.copy()
+    oracle.step(w_plain, g, e1, lr, mode=EF)
+    ghat_mean = (w0.astype(np.float64) - w_plain) / lr
+    w, m, e2 = w0.copy(), np.zeros(n, np.float32), e.copy()
+    oracle.step_momentum(w, m, g, e2, lr, 0.0, wd, mode=EF)
+    assert np.allclose(w, w0.astype(np.float64) * (1 - lr * wd) - lr * ghat_mean, rtol=0, atol=1e-6)
+    assert np.array_equal(e1, e2)
+
+
+@pytest.mark.parametrize("seed", range(12))
+def test_momentum_bruteforce_rational(seed):
+    rng = np.random.default_rng(100 + seed)
+    n = int(rng.integers(1, 17))
+    P = int(rng.integers(1, 5))
+    mode = EF if seed % 2 == 0 else ALG1
+    g = (rng.standard_normal((P, n)) * 10.0 ** rng.uniform(-3, 1)).astype(np.float32)
+    e = (rng.standard_normal((P, n)) * 10.0 ** rng.uniform(-3, 1)).astype(np.float32)
+    lr, beta, wd = np.float32(0.3), np.float32(0.9), np.float32(5e-4)
+    v = (g + e).astype(np.float32) if mode == EF else g
+    lm, _, _ = oracle.encode(g, e if mode == EF else None, mode=mode)
+    gm = oracle.global_average(lm)
+    F = lambda x: Fraction(float(x))
+    ghat = [[None] * n for _ in range(P)]
+    for p in range(P):
+        for i in range(n):
+            mean_vec = F(gm[0]) if v[p, i] >= 0 else -F(gm[1])
+            if mode == EF:
+                ghat[p][i] = mean_vec
+            else:
+                enc = F(lm[p, 0]) if v[p, i] >= 0 else -F(lm[p, 1])
+                ghat[p][i] = F(v[p, i]) - enc + mean_vec
+    w0 = rng.standard_normal(n).astype(np.float32)
+    m0 = rng.standard_normal(n).astype(np.float32)
+    # one shared w: the worker-mean of g_hat drives one momentum vector
+    w, m, e_sh = w0.copy(), m0.copy(), e.copy()
+    oracle.decode_update_momentum(w, m, g, e_sh, lm, gm, lr, beta, wd, mode=mode)
+    for i in range(n):
+        u = sum((ghat[p][i] for p in range(P)), Fraction(0)) / P + F(wd) * F(w0[i])
+        m_new = F(beta) * F(m0[i]) + u
+        assert _ulp_close(m[i], _round32(m_new))
+        assert _ulp_close(w[i], _round32(F(w0[i]) - F(lr) * m_new))
+    # one replica per worker: its own g_hat, its own momentum vector
+    w_r, m_r, e_r = np.tile(w0, (P, 1)), np.tile(m0, (P, 1)), e.copy()
+    oracle.decode_update_momentum(w_r, m_r, g, e_r, lm, gm, lr, beta, wd, mode=mode)
+    for p in range(P):
+        for i in range(n):
+            m_new = F(beta) * F(m0[i]) + ghat[p][i] + F(wd) * F(w0[i])
+            assert _ulp_close(m_r[p, i], _round32(m_new))
+            assert _ulp_close(w_r[p, i], _round32(F(w0[i]) - F(lr) * m_new))
+    assert np.array_equal(e_sh, e_r)
+    # the shared state is the mean of the replica states (the update is linear)
+    assert np.allclose(w, w_r.astype(np.float64).mean(0), rtol=0, atol=1e-6 * max(1.0, float(np.abs(w0).max())))
+    assert np.allclose(m, m_r.astype(np.float64).mean(0), rtol=1e-6, atol=1e-6)
