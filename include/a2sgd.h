@@ -152,6 +152,31 @@ int a2sgd_step(a2sgd_ctx *ctx, float *w, int64_t w_stride,
                const float *grad, int64_t grad_stride,
                float *err, int64_t err_stride, float lr, void *stream);
 
+/* Algorithm 1 lines 4, 6 and 7 with the optimiser the paper's experiments put on top of line 7:
+ * SGD with momentum and weight decay (Section 4.1 and Table 1 list the training policies;
+ * Algorithm 1 line 7 itself prints the plain step and has no counterpart for the two terms).  The
+ * method compresses the gradient only (lines 3-6), so both terms act on the reconstructed gradient:
+ *     u = g_hat + weight_decay * w;   mom <- beta * mom + u;   w <- w - lr * mom
+ * (heavy ball, no dampening, no Nesterov look-ahead, decay folded into the gradient).
+ *   mom          in/out, DEVICE, same layout as w: one vector when w is shared (mom_stride == 0,
+ *                it sees the worker-mean of g_hat), one per worker otherwise (mom_stride >= n);
+ *                zero it before the first step
+ *   beta         0 <= beta < 1;  weight_decay >= 0 (A2SGD_ERR_ARG otherwise)
+ * Everything else as a2sgd_decode_update.  beta = weight_decay = 0 gives the same w as
+ * a2sgd_decode_update and leaves g_hat in mom.  One streaming pass: (12P + 16) bytes per model
+ * element for a shared w, 28P for replicas. */
+int a2sgd_decode_update_momentum(a2sgd_ctx *ctx, float *w, int64_t w_stride, float *mom, int64_t mom_stride,
+                                 const float *grad, int64_t grad_stride, float *err, int64_t err_stride,
+                                 const float *local_means, const float *global_means, float lr,
+                                 float beta, float weight_decay, void *stream);
+
+/* a2sgd_step (Algorithm 1 lines 3-7 for all P workers) with the momentum / weight-decay update
+ * above in place of the plain SGD step.  Always two launches.  Not available on contexts
+ * created with A2SGD_DEFERRED_RESIDUAL. */
+int a2sgd_step_momentum(a2sgd_ctx *ctx, float *w, int64_t w_stride, float *mom, int64_t mom_stride,
+                        const float *grad, int64_t grad_stride, float *err, int64_t err_stride,
+                        float lr, float beta, float weight_decay, void *stream);
+
 /* a2sgd_step with the fresh gradients stored as bfloat16 (the paper remarks that the method
  * "can be further integrated with quantization"; a bfloat16 gradient is the common case of a
  * mixed-precision backward pass).  grad: [P] vectors of n bfloat16 values (raw uint16 bit

@@ -63,6 +63,12 @@ def lib() -> ctypes.CDLL:
         l.a2sgd_decode_update.argtypes = [_vp, _vp, _i64, _vp, _i64, _vp, _i64, _vp, _vp, ctypes.c_float, _vp]
         l.a2sgd_step.restype = ctypes.c_int
         l.a2sgd_step.argtypes = [_vp, _vp, _i64, _vp, _i64, _vp, _i64, ctypes.c_float, _vp]
+        l.a2sgd_decode_update_momentum.restype = ctypes.c_int
+        l.a2sgd_decode_update_momentum.argtypes = [_vp, _vp, _i64, _vp, _i64, _vp, _i64, _vp, _i64, _vp, _vp,
+                                                   ctypes.c_float, ctypes.c_float, ctypes.c_float, _vp]
+        l.a2sgd_step_momentum.restype = ctypes.c_int
+        l.a2sgd_step_momentum.argtypes = [_vp, _vp, _i64, _vp, _i64, _vp, _i64, _vp, _i64,
+                                          ctypes.c_float, ctypes.c_float, ctypes.c_float, _vp]
         l.a2sgd_step_host.restype = ctypes.c_int
         l.a2sgd_step_host.argtypes = [_vp, _vp, _i64, _vp, _i64, _vp, _i64, _vp, _i64, ctypes.c_float, _vp, _vp]
         l.a2sgd_read_stats.restype = ctypes.c_int
@@ -227,6 +233,31 @@ def a2sgd_step(ctx: Context, w: torch.Tensor, grad: torch.Tensor, err: Optional[
     gp, gs = _rows(grad, "grad")
     ep, es = _rows(err, "err")
     _check(lib().a2sgd_step(ctx.handle, wp, ws, gp, gs, ep, es, float(lr), _stream(stream)), "a2sgd_step")
+
+
+def a2sgd_decode_update_momentum(ctx: Context, w: torch.Tensor, mom: torch.Tensor, grad: torch.Tensor,
+                                 err: Optional[torch.Tensor], local_means: Optional[torch.Tensor],
+                                 global_means: torch.Tensor, lr: float, beta: float, weight_decay: float,
+                                 stream=None) -> None:
+    """mom: float32 CUDA tensor with the layout of w (zero before the first step)."""
+    wp, ws = _weights(w)
+    mp, ms = _weights(mom)
+    gp, gs = _rows(grad, "grad")
+    ep, es = _rows(err, "err")
+    _check(lib().a2sgd_decode_update_momentum(ctx.handle, wp, ws, mp, ms, gp, gs, ep, es,
+                                              local_means.data_ptr() if local_means is not None else None,
+                                              global_means.data_ptr(), float(lr), float(beta), float(weight_decay),
+                                              _stream(stream)), "a2sgd_decode_update_momentum")
+
+
+def a2sgd_step_momentum(ctx: Context, w: torch.Tensor, mom: torch.Tensor, grad: torch.Tensor,
+                        err: Optional[torch.Tensor], lr: float, beta: float, weight_decay: float, stream=None) -> None:
+    wp, ws = _weights(w)
+    mp, ms = _weights(mom)
+    gp, gs = _rows(grad, "grad")
+    ep, es = _rows(err, "err")
+    _check(lib().a2sgd_step_momentum(ctx.handle, wp, ws, mp, ms, gp, gs, ep, es, float(lr), float(beta),
+                                     float(weight_decay), _stream(stream)), "a2sgd_step_momentum")
 
 
 def a2sgd_step_bf16(ctx: Context, w: torch.Tensor, grad: torch.Tensor, err: Optional[torch.Tensor], lr: float,

@@ -181,40 +181,58 @@ const void *select_encode(bool ef, bool mask, int vw)
 #undef A2_PICK
 }
 
-template <bool EF, bool STORE, int VW>
+template <bool EF, bool STORE, int VW, bool MOM>
 const void *select_decode_shared_p(uint32_t P)
 {
     switch (P) {
-    case 1: return (const void *)k_decode_shared_vec<EF, STORE, 1, VW>;
-    case 2: return (const void *)k_decode_shared_vec<EF, STORE, 2, VW>;
-    case 4: return (const void *)k_decode_shared_vec<EF, STORE, 4, VW>;
-    case 8: return (const void *)k_decode_shared_vec<EF, STORE, 8, VW>;
-    default: return (const void *)k_decode_shared_vec<EF, STORE, 0, VW>;
+    case 1: return (const void *)k_decode_shared_vec<EF, STORE, 1, VW, 0, MOM>;
+    case 2: return (const void *)k_decode_shared_vec<EF, STORE, 2, VW, 0, MOM>;
+    case 4: return (const void *)k_decode_shared_vec<EF, STORE, 4, VW, 0, MOM>;
+    case 8: return (const void *)k_decode_shared_vec<EF, STORE, 8, VW, 0, MOM>;
+    default: return (const void *)k_decode_shared_vec<EF, STORE, 0, VW, 0, MOM>;
     }
 }
 
-const void *select_decode_shared(bool ef, bool store, uint32_t P, int vw)
+template <bool MOM>
+const void *select_decode_shared_m(bool ef, bool store, uint32_t P, int vw)
 {
     if (vw == 8) {
-        if (ef) return select_decode_shared_p<true, true, 8>(P);
-        return store ? select_decode_shared_p<false, true, 8>(P) : select_decode_shared_p<false, false, 8>(P);
+        if (ef) return select_decode_shared_p<true, true, 8, MOM>(P);
+        return store ? select_decode_shared_p<false, true, 8, MOM>(P) : select_decode_shared_p<false, false, 8, MOM>(P);
     }
-    if (ef) return select_decode_shared_p<true, true, 4>(P);
-    return store ? select_decode_shared_p<false, true, 4>(P) : select_decode_shared_p<false, false, 4>(P);
+    if (ef) return select_decode_shared_p<true, true, 4, MOM>(P);
+    return store ? select_decode_shared_p<false, true, 4, MOM>(P) : select_decode_shared_p<false, false, 4, MOM>(P);
 }
 
-const void *select_decode_repl(bool ef, bool store, int vw)
+const void *select_decode_shared(bool ef, bool store, uint32_t P, int vw, bool mom = false)
+{
+    return mom ? select_decode_shared_m<true>(ef, store, P, vw) : select_decode_shared_m<false>(ef, store, P, vw);
+}
+
+template <bool MOM>
+const void *select_decode_repl_m(bool ef, bool store, int vw)
 {
     if (vw == 8) {
-        if (ef) return (const void *)k_decode_repl_vec<true, true, 8>;
-        return store ? (const void *)k_decode_repl_vec<false, true, 8> : (const void *)k_decode_repl_vec<false, false, 8>;
+        if (ef) return (const void *)k_decode_repl_vec<true, true, 8, 0, MOM>;
+        return store ? (const void *)k_decode_repl_vec<false, true, 8, 0, MOM>
+                     : (const void *)k_decode_repl_vec<false, false, 8, 0, MOM>;
     }
-    if (ef) return (const void *)k_decode_repl_vec<true, true, 4>;
-    return store ? (const void *)k_decode_repl_vec<false, true, 4> : (const void *)k_decode_repl_vec<false, false, 4>;
+    if (ef) return (const void *)k_decode_repl_vec<true, true, 4, 0, MOM>;
+    return store ? (const void *)k_decode_repl_vec<false, true, 4, 0, MOM>
+                 : (const void *)k_decode_repl_vec<false, false, 4, 0, MOM>;
 }
 
-const void *select_decode_scalar(bool ef, bool store)
+const void *select_decode_repl(bool ef, bool store, int vw, bool mom = false)
 {
+    return mom ? select_decode_repl_m<true>(ef, store, vw) : select_decode_repl_m<false>(ef, store, vw);
+}
+
+const void *select_decode_scalar(bool ef, bool store, bool mom = false)
+{
+    if (mom) {
+        if (ef) return (const void *)k_decode_scalar<true, true, 0, true>;
+        return store ? (const void *)k_decode_scalar<false, true, 0, true> : (const void *)k_decode_scalar<false, false, 0, true>;
+    }
     if (ef) return (const void *)k_decode_scalar<true, true>;
     return store ? (const void *)k_decode_scalar<false, true> : (const void *)k_decode_scalar<false, false>;
 }
@@ -387,26 +405,42 @@ int launch_encode(a2sgd_ctx *c, const float *grad, int64_t gs, const float *err,
     return A2SGD_OK;
 }
 
+// Momentum / weight-decay form of the update: the buffer (layout of w) and the two coefficients.
+struct MomentumArgs {
+    float *mom = nullptr;
+    int64_t mom_stride = 0;
+    float beta = 0.f;
+    float weight_decay = 0.f;
+};
+
 int launch_decode(a2sgd_ctx *c, float *w, int64_t ws, const float *grad, int64_t gs, float *err,
                   int64_t es, const float *local_means, const float *global_means, float lr,
-                  cudaStream_t s)
+                  cudaStream_t s, const MomentumArgs *mo = nullptr)
 {
     const bool ef = !c->alg1;
     const bool store = ef || err != nullptr;
     const bool shared = ws == 0;
-    const int vw = decode_vec_width(c, w, ws, grad, gs, err, es);
+    const bool mom = mo != nullptr;
+    int vw = decode_vec_width(c, w, ws, grad, gs, err, es);
+    if (mom) vw = std::min(vw, vec_width(mo->mom, ws == 0 ? 8 : mo->mom_stride, c->P));
     DecodeArgs a = make_decode_args(c, w, ws, grad, gs, err, es, local_means, global_means, lr);
+    if (mom) {
+        a.mom = mo->mom;
+        a.mom_stride = shared ? 0 : mo->mom_stride;
+        a.beta = mo->beta;
+        a.weight_decay = mo->weight_decay;
+    }
     void *params[] = {&a};
     const void *fn;
     dim3 grid;
     if (vw && shared) {
-        fn = select_decode_shared(ef, store, c->P, vw);
+        fn = select_decode_shared(ef, store, c->P, vw, mom);
         grid = dim3(flat_grid(c, occupancy(c, fn), (c->n + vw - 1) / vw, A2SGD_WAVES_K3));
     } else if (vw) {
-        fn = select_decode_repl(ef, store, vw);
+        fn = select_decode_repl(ef, store, vw, mom);
         grid = dim3(per_worker_grid(c, occupancy(c, fn), (c->n + vw - 1) / vw, A2SGD_WAVES_K3), c->P);
     } else {
-        fn = select_decode_scalar(ef, store);
+        fn = select_decode_scalar(ef, store, mom);
         grid = shared ? dim3(flat_grid(c, occupancy(c, fn), c->n, A2SGD_WAVES_K3), 1)
                       : dim3(per_worker_grid(c, occupancy(c, fn), c->n, A2SGD_WAVES_K3), c->P);
     }
@@ -709,6 +743,69 @@ extern "C" int a2sgd_step(a2sgd_ctx *c, float *w, int64_t w_stride, const float 
                                  c->global_means, s);
     if (r1) return r1;
     return launch_decode(c, w, ws, grad, grad_stride, err, err_stride, c->local_means, c->global_means, lr, s);
+}
+
+// Argument checks shared by the two momentum entry points.
+static int check_momentum(const a2sgd_ctx *c, const float *w, int64_t w_stride, const float *mom, int64_t mom_stride,
+                          float beta, float weight_decay)
+{
+    if (!w || !mom) return A2SGD_ERR_ARG;
+    if (c->flags & A2SGD_DEFERRED_RESIDUAL) return A2SGD_ERR_ARG;
+    if (w_stride != 0 && !stride_ok(w_stride, c->n, c->P)) return A2SGD_ERR_ARG;
+    if (c->P > 1 && (w_stride == 0) != (mom_stride == 0)) return A2SGD_ERR_ARG; // same layout as w
+    if (mom_stride != 0 && !stride_ok(mom_stride, c->n, c->P)) return A2SGD_ERR_ARG;
+    if (!(beta >= 0.0f && beta < 1.0f) || !(weight_decay >= 0.0f)) return A2SGD_ERR_ARG;
+    if (!aligned(w, 4) || !aligned(mom, 4)) return A2SGD_ERR_ALIGN;
+    if (!device_pointer_ok(c, w) || !device_pointer_ok(c, mom)) return A2SGD_ERR_ARG;
+    return A2SGD_OK;
+}
+
+extern "C" int a2sgd_decode_update_momentum(a2sgd_ctx *c, float *w, int64_t w_stride, float *mom, int64_t mom_stride,
+                                            const float *grad, int64_t grad_stride, float *err, int64_t err_stride,
+                                            const float *local_means, const float *global_means, float lr,
+                                            float beta, float weight_decay, void *stream)
+{
+    if (!c || !global_means) return A2SGD_ERR_ARG;
+    int rc = check_common(c, grad, grad_stride, err, err_stride, !c->alg1);
+    if (rc) return rc;
+    rc = check_momentum(c, w, w_stride, mom, mom_stride, beta, weight_decay);
+    if (rc) return rc;
+    if (c->alg1 && !local_means) return A2SGD_ERR_ARG;
+    if (!aligned(global_means, 4) || (local_means && !aligned(local_means, 4))) return A2SGD_ERR_ALIGN;
+    if (!device_pointer_ok(c, global_means) || !device_pointer_ok(c, local_means)) return A2SGD_ERR_ARG;
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return A2SGD_ERR_CUDA;
+    MomentumArgs mo;
+    mo.mom = mom;
+    mo.mom_stride = mom_stride;
+    mo.beta = beta;
+    mo.weight_decay = weight_decay;
+    return launch_decode(c, w, (c->P == 1) ? 0 : w_stride, grad, grad_stride, err, err_stride, local_means,
+                         global_means, lr, static_cast<cudaStream_t>(stream), &mo);
+}
+
+extern "C" int a2sgd_step_momentum(a2sgd_ctx *c, float *w, int64_t w_stride, float *mom, int64_t mom_stride,
+                                   const float *grad, int64_t grad_stride, float *err, int64_t err_stride,
+                                   float lr, float beta, float weight_decay, void *stream)
+{
+    if (!c) return A2SGD_ERR_ARG;
+    int rc = check_common(c, grad, grad_stride, err, err_stride, !c->alg1);
+    if (rc) return rc;
+    rc = check_momentum(c, w, w_stride, mom, mom_stride, beta, weight_decay);
+    if (rc) return rc;
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return A2SGD_ERR_CUDA;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    MomentumArgs mo;
+    mo.mom = mom;
+    mo.mom_stride = mom_stride;
+    mo.beta = beta;
+    mo.weight_decay = weight_decay;
+    const int r1 = launch_encode(c, grad, grad_stride, err, err_stride, c->local_means, c->pos_counts, nullptr,
+                                 c->global_means, s);
+    if (r1) return r1;
+    return launch_decode(c, w, (c->P == 1) ? 0 : w_stride, grad, grad_stride, err, err_stride, c->local_means,
+                         c->global_means, lr, s, &mo);
 }
 
 static int step_lowp(a2sgd_ctx *c, float *w, int64_t w_stride, const uint16_t *grad, int64_t grad_stride,

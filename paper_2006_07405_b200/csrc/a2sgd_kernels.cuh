@@ -580,7 +580,53 @@ struct DecodeArgs {
     const float *local_means;  // [P][2] (ALG1)
     const float *global_means; // [2]
     float lr;
+    // momentum / weight-decay form of the update (MOM kernels only); mom has the layout of w
+    float *mom;
+    int64_t mom_stride;
+    float beta;
+    float weight_decay;
 };
+
+// The update applied to one weight once its reconstructed gradient is known.
+//   plain (Algorithm 1 line 7):  w <- w + scale * g_sum          (scale = -lr, or -lr/P for a shared w)
+//   MOM (heavy-ball momentum and weight decay acting on the reconstructed gradient):
+//        u = g_sum / p + wd * w;   m <- beta * m + u;   w <- w - lr * m
+struct UpdateConst {
+    float scale;  // plain form
+    float p;      // MOM: divisor of g_sum (1 for a replica, P for a shared w)
+    float beta, wd, neg_lr;
+};
+
+template <bool MOM>
+__device__ __forceinline__ float update1(const UpdateConst &u, float g_sum, float w, float &m)
+{
+    if (MOM) {
+        const float gbar = u.p == 1.0f ? g_sum : g_sum / u.p;
+        m = fmaf(u.beta, m, fmaf(u.wd, w, gbar));
+        return fmaf(u.neg_lr, m, w);
+    }
+    return fmaf(u.scale, g_sum, w);
+}
+
+template <bool MOM, int VW>
+__device__ __forceinline__ Vec<VW> update_vec(const UpdateConst &u, const Vec<VW> &g_sum, const Vec<VW> &w, Vec<VW> &m)
+{
+    Vec<VW> r;
+#pragma unroll
+    for (int k = 0; k < VW; ++k) r.v[k] = update1<MOM>(u, g_sum.v[k], w.v[k], m.v[k]);
+    return r;
+}
+
+__device__ __forceinline__ UpdateConst update_const(const DecodeArgs &a, float divisor)
+{
+    UpdateConst u;
+    u.scale = -a.lr / divisor;
+    u.p = divisor;
+    u.beta = a.beta;
+    u.wd = a.weight_decay;
+    u.neg_lr = -a.lr;
+    return u;
+}
 
 // Per-worker constants of the reconstruction.
 //   EF  : g_hat = pos ? m_pos : -m_neg                      e' = v - g_hat
@@ -653,7 +699,7 @@ __device__ __forceinline__ Vec<VW> zero_vec()
 // workers in order (fixed summation order), so w is read and written once
 // per model element.  PT > 0: P known at compile time (all 2P+1 loads of a
 // vector are issued before any is used); PT == 0: run-time P.
-template <bool EF, bool STORE, int PT, int VW, int GB = 0>
+template <bool EF, bool STORE, int PT, int VW, int GB = 0, bool MOM = false>
 __global__ void __launch_bounds__(kBlock) k_decode_shared_vec(DecodeArgs a)
 {
     pdl_wait_prior_grid();
@@ -662,7 +708,7 @@ __global__ void __launch_bounds__(kBlock) k_decode_shared_vec(DecodeArgs a)
     __shared__ WorkerConst sh_c[PT > 0 ? 1 : kMaxP];
     const uint32_t P = PT > 0 ? PT : a.P;
     const float m_pos = __ldg(a.global_means), m_neg = __ldg(a.global_means + 1);
-    const float scale = -a.lr / (float)P;
+    const UpdateConst uc = update_const(a, (float)P);
     const uint64_t nv = a.n / VW;
     const uint64_t stride = (uint64_t)gridDim.x * kBlock;
 
@@ -676,6 +722,7 @@ __global__ void __launch_bounds__(kBlock) k_decode_shared_vec(DecodeArgs a)
             // (6.55 -> 6.77 TB/s): fewer concurrent streams per thread, lower register count
             constexpr int PB = PP < 4 ? PP : 4;
             const Vec<VW> wv = ld_vec<VW>(a.w + VW * j);
+            Vec<VW> mv = MOM ? ld_vec<VW>(a.mom + VW * j) : zero_vec<VW>();
             Vec<VW> sum = zero_vec<VW>();
 #pragma unroll
             for (int p0 = 0; p0 < PP; p0 += PB) {
@@ -697,13 +744,15 @@ __global__ void __launch_bounds__(kBlock) k_decode_shared_vec(DecodeArgs a)
                     if (STORE) st_vec<VW>(a.err + (int64_t)(p0 + q) * a.err_stride + VW * j, rs);
                 }
             }
-            st_vec<VW>(a.w + VW * j, axpy_vec<VW>(scale, sum, wv));
+            st_vec<VW>(a.w + VW * j, update_vec<MOM, VW>(uc, sum, wv, mv));
+            if (MOM) st_vec<VW>(a.mom + VW * j, mv);
         }
     } else {
         for (uint32_t p = threadIdx.x; p < P; p += kBlock) sh_c[p] = worker_const<EF>(a, p, m_pos, m_neg);
         __syncthreads();
         for (uint64_t j = (uint64_t)blockIdx.x * kBlock + threadIdx.x; j < nv; j += stride) {
             const Vec<VW> wv = ld_vec<VW>(a.w + VW * j);
+            Vec<VW> mv = MOM ? ld_vec<VW>(a.mom + VW * j) : zero_vec<VW>();
             Vec<VW> sum = zero_vec<VW>();
             for (uint32_t p = 0; p < P; ++p) {
                 Vec<VW> v = GradRow<GB>(a.grad, (int64_t)p * a.grad_stride).template vec<VW>(VW * j);
@@ -713,7 +762,8 @@ __global__ void __launch_bounds__(kBlock) k_decode_shared_vec(DecodeArgs a)
                 sum = add_vec<VW>(sum, gh);
                 if (STORE) st_vec<VW>(a.err + (int64_t)p * a.err_stride + VW * j, rs);
             }
-            st_vec<VW>(a.w + VW * j, axpy_vec<VW>(scale, sum, wv));
+            st_vec<VW>(a.w + VW * j, update_vec<MOM, VW>(uc, sum, wv, mv));
+            if (MOM) st_vec<VW>(a.mom + VW * j, mv);
         }
     }
     // the n % VW trailing elements
@@ -730,13 +780,15 @@ __global__ void __launch_bounds__(kBlock) k_decode_shared_vec(DecodeArgs a)
                 sum += gh;
                 if (STORE) st_stream1(a.err + (int64_t)p * a.err_stride + i, rs);
             }
-            a.w[i] = fmaf(scale, sum, a.w[i]);
+            float m = MOM ? a.mom[i] : 0.f;
+            a.w[i] = update1<MOM>(uc, sum, a.w[i], m);
+            if (MOM) a.mom[i] = m;
         }
     }
 }
 
 // One w replica per worker (Algorithm 1's layout).  grid = (G, P).
-template <bool EF, bool STORE, int VW, int GB = 0>
+template <bool EF, bool STORE, int VW, int GB = 0, bool MOM = false>
 __global__ void __launch_bounds__(kBlock) k_decode_repl_vec(DecodeArgs a)
 {
     pdl_wait_prior_grid();
@@ -748,13 +800,14 @@ __global__ void __launch_bounds__(kBlock) k_decode_repl_vec(DecodeArgs a)
     const GradRow<GB> g(a.grad, (int64_t)p * a.grad_stride);
     float *e = (EF || STORE) ? a.err + (int64_t)p * a.err_stride : nullptr;
     float *w = a.w + (int64_t)p * a.w_stride;
-    const float neg_lr = -a.lr;
+    float *mom = MOM ? a.mom + (int64_t)p * a.mom_stride : nullptr;
+    const UpdateConst uc = update_const(a, 1.0f);
     const uint64_t nv = a.n / VW;
     const uint64_t stride = (uint64_t)gridDim.x * kBlock;
     uint64_t j = (uint64_t)blockIdx.x * kBlock + threadIdx.x;
     constexpr int U = 8 / VW;
     for (; j + (U - 1) * stride < nv; j += U * stride) {
-        Vec<VW> gv[U], ev[U], wv[U];
+        Vec<VW> gv[U], ev[U], wv[U], mv[U];
 #pragma unroll
         for (int u = 0; u < U; ++u) gv[u] = g.template vec<VW>(VW * (j + u * stride));
         if (EF) {
@@ -764,22 +817,27 @@ __global__ void __launch_bounds__(kBlock) k_decode_repl_vec(DecodeArgs a)
 #pragma unroll
         for (int u = 0; u < U; ++u) wv[u] = ld_vec<VW>(w + VW * (j + u * stride));
 #pragma unroll
+        for (int u = 0; u < U; ++u) mv[u] = MOM ? ld_vec<VW>(mom + VW * (j + u * stride)) : zero_vec<VW>();
+#pragma unroll
         for (int u = 0; u < U; ++u) {
             const Vec<VW> v = EF ? add_vec<VW>(gv[u], ev[u]) : gv[u];
             Vec<VW> gh, rs;
             decode_vec<EF, VW>(v, c, gh, rs);
             if (STORE) st_vec<VW>(e + VW * (j + u * stride), rs);
-            st_vec<VW>(w + VW * (j + u * stride), axpy_vec<VW>(neg_lr, gh, wv[u]));
+            st_vec<VW>(w + VW * (j + u * stride), update_vec<MOM, VW>(uc, gh, wv[u], mv[u]));
+            if (MOM) st_vec<VW>(mom + VW * (j + u * stride), mv[u]);
         }
     }
     for (; j < nv; j += stride) {
         Vec<VW> v = g.template vec<VW>(VW * j);
         if (EF) v = add_vec<VW>(v, ld_vec<VW>(e + VW * j));
         const Vec<VW> wv = ld_vec<VW>(w + VW * j);
+        Vec<VW> mv = MOM ? ld_vec<VW>(mom + VW * j) : zero_vec<VW>();
         Vec<VW> gh, rs;
         decode_vec<EF, VW>(v, c, gh, rs);
         if (STORE) st_vec<VW>(e + VW * j, rs);
-        st_vec<VW>(w + VW * j, axpy_vec<VW>(neg_lr, gh, wv));
+        st_vec<VW>(w + VW * j, update_vec<MOM, VW>(uc, gh, wv, mv));
+        if (MOM) st_vec<VW>(mom + VW * j, mv);
     }
     if (blockIdx.x == 0 && threadIdx.x < VW) {
         const uint64_t i = nv * VW + threadIdx.x;
@@ -789,14 +847,16 @@ __global__ void __launch_bounds__(kBlock) k_decode_repl_vec(DecodeArgs a)
             float gh, rs;
             decode1<EF>(v, c, gh, rs);
             if (STORE) st_stream1(e + i, rs);
-            w[i] = fmaf(neg_lr, gh, w[i]);
+            float m = MOM ? mom[i] : 0.f;
+            w[i] = update1<MOM>(uc, gh, w[i], m);
+            if (MOM) mom[i] = m;
         }
     }
 }
 
 // General path: any 4-byte alignment, both weight layouts, scalar accesses.
 // Shared w: grid = (G, 1), the thread walks the workers; replicas: grid = (G, P).
-template <bool EF, bool STORE, int GB = 0>
+template <bool EF, bool STORE, int GB = 0, bool MOM = false>
 __global__ void __launch_bounds__(kBlock) k_decode_scalar(DecodeArgs a)
 {
     pdl_wait_prior_grid();
@@ -806,7 +866,7 @@ __global__ void __launch_bounds__(kBlock) k_decode_scalar(DecodeArgs a)
     const uint64_t stride = (uint64_t)gridDim.x * kBlock;
     const bool shared = a.w_stride == 0;
     const uint32_t p_lo = shared ? 0 : blockIdx.y, p_hi = shared ? a.P : blockIdx.y + 1;
-    const float scale = shared ? -a.lr / (float)a.P : -a.lr;
+    const UpdateConst uc = update_const(a, shared ? (float)a.P : 1.0f);
     for (uint64_t i = (uint64_t)blockIdx.x * kBlock + threadIdx.x; i < a.n; i += stride) {
         float sum = 0.f;
         for (uint32_t p = p_lo; p < p_hi; ++p) {
@@ -819,7 +879,10 @@ __global__ void __launch_bounds__(kBlock) k_decode_scalar(DecodeArgs a)
             if (STORE) st_stream1(a.err + (int64_t)p * a.err_stride + i, rs);
         }
         float *wp = a.w + (int64_t)p_lo * a.w_stride + i;
-        *wp = fmaf(scale, sum, *wp);
+        float *mp = MOM ? a.mom + (int64_t)p_lo * a.mom_stride + i : nullptr;
+        float m = MOM ? *mp : 0.f;
+        *wp = update1<MOM>(uc, sum, *wp, m);
+        if (MOM) *mp = m;
     }
 }
 
