@@ -22,6 +22,9 @@ and says so in ``config``.  The smaller configurations are timed too and reporte
 
 With N > 1 (under torchrun) every rank runs an independent replica of the workload on its own
 GPU — the benchmarked path has no exchange between GPUs — and the time is the max over ranks.
+A second leg (``exchange_between_gpus``) then runs the method as Algorithm 1 prints it, one worker
+per GPU, and times the exchange of the two local means over NCCL both ways: all-gather plus a
+local fixed-order average, and all-reduce plus division.
 """
 from __future__ import annotations
 
@@ -539,6 +542,100 @@ def next_rows_of(wl, res, peak_gbs) -> dict:
     return rows
 
 
+class DeviceTimer:
+    """CUDA-event stopwatch on the current stream of ``dev``."""
+
+    def __init__(self, dev):
+        import torch
+        self.torch, self.dev = torch, dev
+
+    def mark(self):
+        ev = self.torch.cuda.Event(enable_timing=True)
+        ev.record()
+        return ev
+
+    def sync(self):
+        self.torch.cuda.synchronize(self.dev)
+
+    def ms(self, a, b):
+        return a.elapsed_time(b)
+
+
+class HostTimer:
+    """Wall-clock stand-in with the same interface (CPU tests of the multi-rank protocol)."""
+
+    def __init__(self, dev=None):
+        self.dev = dev
+
+    def mark(self):
+        return time.perf_counter()
+
+    def sync(self):
+        pass
+
+    def ms(self, a, b):
+        return (b - a) * 1e3
+
+
+def exchange_leg(sizes, make_case, dist, dev, steps, warmup, timer):
+    """One worker per rank, as Algorithm 1 prints it: for every n in ``sizes`` and both exchanges
+    of the two local means (all-gather + local fixed-order average; all-reduce + division), times
+    the whole step (encode, exchange, decode/update) and the exchange alone, K calls each,
+    bracketed by barriers, max over ranks.  ``make_case(n, exchange)`` returns (worker, step_call)
+    where ``worker.exchange_means()`` is the exchange alone and ``step_call()`` one whole step."""
+    def barrier():
+        timer.sync()
+        dist.barrier()
+        timer.sync()
+
+    out = {"workers": dist.get_world_size(), "payload_bytes_per_worker": 8, "sizes": {}}
+    for n in sizes:
+        row = {}
+        for exchange in ("allgather", "allreduce"):
+            worker, step_call = make_case(n, exchange)
+            for _ in range(max(3, warmup)):
+                step_call()
+            barrier()
+            t0 = timer.mark()
+            for _ in range(steps):
+                step_call()
+            t1 = timer.mark()
+            barrier()
+            step_ms = max_over_ranks(timer.ms(t0, t1), dist, dev) / steps
+            for _ in range(max(3, warmup)):
+                worker.exchange_means()
+            barrier()
+            reps = max(steps, 50)
+            t0 = timer.mark()
+            for _ in range(reps):
+                worker.exchange_means()
+            t1 = timer.mark()
+            barrier()
+            ex_us = max_over_ranks(timer.ms(t0, t1), dist, dev) / reps * 1e3
+            row[exchange] = {"ms_per_step": step_ms, "us_per_exchange": ex_us,
+                             "worker_params_per_s": dist.get_world_size() * n / (step_ms * 1e-3)}
+            worker.destroy()
+        out["sizes"][str(n)] = row
+    return out
+
+
+def device_exchange_case(dev, lr):
+    """make_case for exchange_leg on GPUs: DistributedA2SGD with seeded per-rank gradients."""
+    import torch
+    from paper_2006_07405_b200 import binding as B
+    from paper_2006_07405_b200 import distributed as D
+
+    def make(n, exchange):
+        import torch.distributed as dist_mod
+        gen = torch.Generator(device=dev).manual_seed(20060740 + dist_mod.get_rank())
+        g = B.padded_rows(1, n, dev).normal_(0.0, 1e-3, generator=gen)
+        e = B.padded_rows(1, n, dev, fill=0.0)
+        w = torch.zeros(n, device=dev)
+        worker = D.DistributedA2SGD(n, dev.index, B.MODE_EF, exchange=exchange)
+        return worker, (lambda: worker.step(w, g, e, lr))
+    return make
+
+
 def pick_workload(name, scale_div, dev):
     """The requested workload, or the fallback when the device cannot hold its resident set."""
     import torch
@@ -565,6 +662,8 @@ def main():
     ap.add_argument("--impl", default="native", choices=["native", "reference"])
     ap.add_argument("--no-extra", action="store_true", help="skip the other configurations at N=1")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--exchange-leg", action="store_true",
+                    help="under torchrun: run the one-worker-per-GPU exchange leg even with a single rank")
     ap.add_argument("--scale-div", type=int, default=1,
                     help="divide every tensor length of the workload (small cases for profiler captures)")
     ap.add_argument("--variant", default="step",
@@ -643,6 +742,11 @@ def main():
             r2 = time_workload(w2, k, 3, dev, with_e2e=False)
             extra[name] = summarise(w2, r2, 1, peak_gbs)
 
+    exchange = None
+    if dist is not None and ((world > 1 and not args.no_extra) or args.exchange_leg):
+        # the O(1) exchange between real GPUs (Algorithm 1 line 5), all-gather against all-reduce
+        sizes = sorted({1 << 20, W.get_workload("c2_lstm_ptb").n, wl.n})
+        exchange = exchange_leg(sizes, device_exchange_case(dev, wl.lr), dist, dev, steps, warmup, DeviceTimer(dev))
     if dist is not None:
         dist.barrier()
     if rank != 0:
@@ -692,6 +796,8 @@ def main():
         line["next_rows"] = rows
     if extra:
         line["other_workloads"] = extra
+    if exchange:
+        line["exchange_between_gpus"] = exchange
     if not args.no_cpu_baseline and world == 1:
         cb = oracle_sample_rate(wl, 10.0)
         line["cpu_baseline"] = dict({k: v for k, v in cb.items() if not k.startswith("_")}, host=host_description())

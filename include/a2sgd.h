@@ -130,6 +130,16 @@ int a2sgd_encode(a2sgd_ctx *ctx, const float *grad, int64_t grad_stride,
 int a2sgd_global_average(a2sgd_ctx *ctx, const float *local_means,
                          float *global_means, void *stream);
 
+/* Algorithm 1 line 5 with one worker per GPU, for an exchange done as the paper does it, by
+ * Allreduce: a collective between the GPUs has formed the SUMS of the two local means over all
+ * workers (in fp64, so that the order in which the collective adds cannot matter at fp32
+ * precision); this call divides by the worker count in fp64 and rounds once — the "average" of
+ * Allreduce(average), inside the library.
+ *   sums  in, DEVICE, [2] doubles = {sum_p mu_pos^p, sum_p mu_neg^p};  workers >= 1
+ *   global_means  out, [2] */
+int a2sgd_global_average_from_sums(a2sgd_ctx *ctx, const double *sums, uint32_t workers,
+                                   float *global_means, void *stream);
+
 /* Algorithm 1 lines 4, 6 and 7 fused: reconstruct, update the residual,
  * apply the SGD step.  Reads grad, err (EF) and w once, writes err and w once.
  *   w            in/out; w_stride == 0: one shared vector, else >= n: one per worker
@@ -209,6 +219,14 @@ int a2sgd_materialize_err(a2sgd_ctx *ctx, float *err, int64_t err_stride, void *
  * (4P + 8) bytes per model element for a shared w. */
 int a2sgd_dense_sync(a2sgd_ctx *ctx, float *w, int64_t w_stride,
                      const float *grad, int64_t grad_stride, float lr, void *stream);
+
+/* Algorithm 1 lines 9-10 with one worker per GPU: the dense Allreduce between the GPUs has
+ * already formed grad_sum, the element-wise SUM of all workers' gradients; this call applies
+ * w <- w - lr * grad_sum / workers (the division that makes the all-reduce an average is done
+ * here, not by the caller).  Contexts with P == 1 only (this rank's one worker).
+ *   grad_sum  in, DEVICE, [n];  workers >= 1 */
+int a2sgd_dense_sync_reduced(a2sgd_ctx *ctx, float *w, const float *grad_sum, uint32_t workers, float lr,
+                             void *stream);
 
 /* Segment lists: the model as S separate tensors (the way a training framework holds its
  * parameters and gradients) instead of one flat vector.  The S tensors are treated as the

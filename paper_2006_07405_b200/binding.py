@@ -69,6 +69,10 @@ def lib() -> ctypes.CDLL:
         l.a2sgd_step_momentum.restype = ctypes.c_int
         l.a2sgd_step_momentum.argtypes = [_vp, _vp, _i64, _vp, _i64, _vp, _i64, _vp, _i64,
                                           ctypes.c_float, ctypes.c_float, ctypes.c_float, _vp]
+        l.a2sgd_global_average_from_sums.restype = ctypes.c_int
+        l.a2sgd_global_average_from_sums.argtypes = [_vp, _vp, ctypes.c_uint32, _vp, _vp]
+        l.a2sgd_dense_sync_reduced.restype = ctypes.c_int
+        l.a2sgd_dense_sync_reduced.argtypes = [_vp, _vp, _vp, ctypes.c_uint32, ctypes.c_float, _vp]
         l.a2sgd_step_host.restype = ctypes.c_int
         l.a2sgd_step_host.argtypes = [_vp, _vp, _i64, _vp, _i64, _vp, _i64, _vp, _i64, ctypes.c_float, _vp, _vp]
         l.a2sgd_read_stats.restype = ctypes.c_int
@@ -213,6 +217,25 @@ def a2sgd_encode_noalloc(grad: torch.Tensor, err: Optional[torch.Tensor], local_
 def a2sgd_global_average(ctx: Context, local_means: torch.Tensor, global_means: torch.Tensor, stream=None) -> None:
     _check(lib().a2sgd_global_average(ctx.handle, local_means.data_ptr(), global_means.data_ptr(), _stream(stream)),
            "a2sgd_global_average")
+
+
+def a2sgd_global_average_from_sums(ctx: Context, sums: torch.Tensor, workers: int, global_means: torch.Tensor,
+                                   stream=None) -> None:
+    """sums: float64 CUDA [2], the all-reduced sums of the two local means over ``workers`` workers."""
+    if sums.dtype != torch.float64 or not sums.is_cuda or sums.numel() < 2:
+        raise ValueError("sums: need a float64 CUDA tensor of 2 elements")
+    _check(lib().a2sgd_global_average_from_sums(ctx.handle, sums.data_ptr(), int(workers), global_means.data_ptr(),
+                                                _stream(stream)), "a2sgd_global_average_from_sums")
+
+
+def a2sgd_dense_sync_reduced(ctx: Context, w: torch.Tensor, grad_sum: torch.Tensor, workers: int, lr: float,
+                             stream=None) -> None:
+    """grad_sum: float32 CUDA [n], the all-reduced sum of the workers' gradients."""
+    if grad_sum.dtype != torch.float32 or not grad_sum.is_cuda or not grad_sum.is_contiguous():
+        raise ValueError("grad_sum: need a contiguous float32 CUDA tensor")
+    wp, _ = _weights(w)
+    _check(lib().a2sgd_dense_sync_reduced(ctx.handle, wp, grad_sum.data_ptr(), int(workers), float(lr),
+                                          _stream(stream)), "a2sgd_dense_sync_reduced")
 
 
 def a2sgd_decode_update(ctx: Context, w: torch.Tensor, grad: torch.Tensor, err: Optional[torch.Tensor],

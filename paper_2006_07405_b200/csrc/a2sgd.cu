@@ -688,10 +688,25 @@ extern "C" int a2sgd_global_average(a2sgd_ctx *c, const float *local_means, floa
 {
     if (!c || !local_means || !global_means) return A2SGD_ERR_ARG;
     if (!aligned(local_means, 4) || !aligned(global_means, 4)) return A2SGD_ERR_ALIGN;
+    if (!device_pointer_ok(c, local_means) || !device_pointer_ok(c, global_means)) return A2SGD_ERR_ARG;
     DeviceGuard guard(c->device);
     if (!guard.ok) return A2SGD_ERR_CUDA;
     k_global_average<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(local_means, c->P, global_means,
                                                                      c->global_means);
+    A2_CUDA(cudaGetLastError());
+    return A2SGD_OK;
+}
+
+extern "C" int a2sgd_global_average_from_sums(a2sgd_ctx *c, const double *sums, uint32_t workers,
+                                              float *global_means, void *stream)
+{
+    if (!c || !sums || !global_means || workers == 0) return A2SGD_ERR_ARG;
+    if (!aligned(sums, 8) || !aligned(global_means, 4)) return A2SGD_ERR_ALIGN;
+    if (!device_pointer_ok(c, sums) || !device_pointer_ok(c, global_means)) return A2SGD_ERR_ARG;
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return A2SGD_ERR_CUDA;
+    k_global_average_from_sums<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(sums, workers, global_means,
+                                                                                c->global_means);
     A2_CUDA(cudaGetLastError());
     return A2SGD_OK;
 }
@@ -882,8 +897,25 @@ extern "C" int a2sgd_materialize_err(a2sgd_ctx *c, float *err, int64_t err_strid
     return A2SGD_OK;
 }
 
+static int dense_sync_impl(a2sgd_ctx *c, float *w, int64_t w_stride, const float *grad, int64_t grad_stride,
+                           float lr, float divisor, void *stream);
+
 extern "C" int a2sgd_dense_sync(a2sgd_ctx *c, float *w, int64_t w_stride, const float *grad, int64_t grad_stride,
                                float lr, void *stream)
+{
+    if (!c) return A2SGD_ERR_ARG;
+    return dense_sync_impl(c, w, w_stride, grad, grad_stride, lr, (float)c->P, stream);
+}
+
+extern "C" int a2sgd_dense_sync_reduced(a2sgd_ctx *c, float *w, const float *grad_sum, uint32_t workers, float lr,
+                                       void *stream)
+{
+    if (!c || c->P != 1 || workers == 0) return A2SGD_ERR_ARG;
+    return dense_sync_impl(c, w, 0, grad_sum, 0, lr, (float)workers, stream);
+}
+
+static int dense_sync_impl(a2sgd_ctx *c, float *w, int64_t w_stride, const float *grad, int64_t grad_stride,
+                           float lr, float divisor, void *stream)
 {
     if (!c || !w || !grad) return A2SGD_ERR_ARG;
     if (!stride_ok(grad_stride, c->n, c->P)) return A2SGD_ERR_ARG;
@@ -902,6 +934,7 @@ extern "C" int a2sgd_dense_sync(a2sgd_ctx *c, float *w, int64_t w_stride, const 
     a.n = c->n;
     a.P = c->P;
     a.lr = lr;
+    a.divisor = divisor;
     const void *fn = select_dense(c->P, vw, ws != 0);
     const uint64_t items = vw ? (c->n + vw - 1) / vw : c->n;
     const dim3 grid(flat_grid(c, occupancy(c, fn), items, A2SGD_WAVES_K3));

@@ -567,6 +567,23 @@ static __global__ void k_global_average(const float *__restrict__ local_means, u
     }
 }
 
+// Algorithm 1 line 5 when the workers sit on different GPUs and a collective has already formed
+// the sums of the two means over all workers (fp64): divide by the worker count, round once.
+static __global__ void k_global_average_from_sums(const double *__restrict__ sums, uint32_t workers,
+                                                  float *global_means, float *ctx_global_means)
+{
+    pdl_wait_prior_grid();
+    pdl_release_next_grid();
+    if (threadIdx.x != 0 || blockIdx.x != 0) return;
+    const float m_pos = (float)(sums[0] / (double)workers), m_neg = (float)(sums[1] / (double)workers);
+    global_means[0] = m_pos;
+    global_means[1] = m_neg;
+    if (ctx_global_means && ctx_global_means != global_means) {
+        ctx_global_means[0] = m_pos;
+        ctx_global_means[1] = m_neg;
+    }
+}
+
 // ------------------------------------------------------------------ K3: decode + residual + SGD
 struct DecodeArgs {
     float *w;
@@ -1006,8 +1023,9 @@ struct DenseArgs {
     const float *grad;
     int64_t grad_stride;
     uint64_t n;
-    uint32_t P;
+    uint32_t P;       // gradient rows summed here
     float lr;
+    float divisor;    // workers the mean is taken over: P, or more when the rows are already sums over ranks
 };
 
 template <int PT, int VW, bool REPL>
@@ -1016,7 +1034,7 @@ __global__ void __launch_bounds__(kBlock) k_dense_sync_vec(DenseArgs a)
     pdl_wait_prior_grid();
     pdl_release_next_grid();
     const uint32_t P = PT > 0 ? PT : a.P;
-    const float scale = -a.lr / (float)P;
+    const float scale = -a.lr / a.divisor;
     const uint64_t nv = a.n / VW;
     const uint64_t stride = (uint64_t)gridDim.x * kBlock;
     for (uint64_t j = (uint64_t)blockIdx.x * kBlock + threadIdx.x; j < nv; j += stride) {
@@ -1059,7 +1077,7 @@ __global__ void __launch_bounds__(kBlock) static k_dense_sync_scalar(DenseArgs a
 {
     pdl_wait_prior_grid();
     pdl_release_next_grid();
-    const float scale = -a.lr / (float)a.P;
+    const float scale = -a.lr / a.divisor;
     const uint64_t stride = (uint64_t)gridDim.x * kBlock;
     const uint32_t reps = a.w_stride == 0 ? 1 : a.P;
     for (uint64_t i = (uint64_t)blockIdx.x * kBlock + threadIdx.x; i < a.n; i += stride) {

@@ -9,13 +9,15 @@ the transport:
 * ``exchange="allgather"`` (default): every rank gathers all 2W scalars and averages them itself
   with the library's fixed-order fp64 kernel, so all ranks hold bit-identical global means.  The
   paper names all-gather as the alternative it expects to be faster than its all-reduce.
-* ``exchange="allreduce"``: the paper's own choice, Allreduce(average) of the two means.
+* ``exchange="allreduce"``: the paper's own choice, Allreduce(average) of the two means: the
+  collective sums the pairs (widened to fp64, so its summation order cannot show at fp32
+  precision) and the library divides by the worker count and rounds once.
 
 With the NCCL backend the two scalars never leave the device.  With gloo (used by the tests) they
 take a round trip through host memory.
 
 The benchmarked configuration of this repository simulates the P workers on ONE GPU and needs none
-of this; a multi-GPU latency study of the two exchanges is not part of this build.
+of this; ``bench.py --gpus N`` (N > 1) additionally times both exchanges with one worker per GPU.
 """
 from __future__ import annotations
 
@@ -37,13 +39,13 @@ def exchange_local_means(local_means: torch.Tensor, group=None) -> torch.Tensor:
     return out if on_device else out.to(local_means.device)
 
 
-def average_local_means(local_means: torch.Tensor, group=None) -> torch.Tensor:
-    """Allreduce(average) of the [P_local, 2] local means (P_local must be 1) -> [2]."""
-    world = dist.get_world_size(group)
+def sum_local_means(local_means: torch.Tensor, group=None) -> torch.Tensor:
+    """All-reduce (SUM) of the [1, 2] local means widened to float64 -> [2] float64 sums over the
+    ranks.  Only the transport happens here; the division that turns the sum into the paper's
+    Allreduce(average) is done by the library (a2sgd_global_average_from_sums)."""
     on_device = local_means.is_cuda and dist.get_backend(group) == "nccl"
-    buf = local_means.reshape(-1).clone() if on_device else local_means.detach().cpu().reshape(-1).clone()
+    buf = local_means.reshape(-1).to(torch.float64) if on_device else local_means.detach().cpu().reshape(-1).to(torch.float64)
     dist.all_reduce(buf, op=dist.ReduceOp.SUM, group=group)
-    buf /= world
     return buf if on_device else buf.to(local_means.device)
 
 
@@ -64,18 +66,24 @@ class DistributedA2SGD:
         self.global_means = torch.zeros(2, device=dev)
         self.pos_count = torch.zeros(1, dtype=torch.int64, device=dev)
 
-    def step(self, w: torch.Tensor, grad: torch.Tensor, err: Optional[torch.Tensor], lr: float) -> None:
-        """Algorithm 1 lines 3-7 at this worker.  w: [n]; grad, err: [1, n] (err None only in ALG1 mode)."""
-        B.a2sgd_encode(self.local, grad, err, self.local_means, self.pos_count)
+    def exchange_means(self) -> None:
+        """Algorithm 1 line 5: this rank's ``local_means`` -> every rank's ``global_means``."""
         if self.exchange == "allgather":
             gathered = exchange_local_means(self.local_means, self.group)
             B.a2sgd_global_average(self.avg, gathered, self.global_means)
         else:
-            self.global_means.copy_(average_local_means(self.local_means, self.group))
+            sums = sum_local_means(self.local_means, self.group)
+            B.a2sgd_global_average_from_sums(self.local, sums, self.world, self.global_means)
+
+    def step(self, w: torch.Tensor, grad: torch.Tensor, err: Optional[torch.Tensor], lr: float) -> None:
+        """Algorithm 1 lines 3-7 at this worker.  w: [n]; grad, err: [1, n] (err None only in ALG1 mode)."""
+        B.a2sgd_encode(self.local, grad, err, self.local_means, self.pos_count)
+        self.exchange_means()
         B.a2sgd_decode_update(self.local, w, grad, err, self.local_means, self.global_means, lr)
 
     def dense_sync(self, w: torch.Tensor, grad: torch.Tensor, lr: float) -> None:
-        """Algorithm 1 lines 9-10: dense all-reduce (average) of the gradient, then the SGD step."""
+        """Algorithm 1 lines 9-10: dense all-reduce of the gradient, then the SGD step with the
+        all-reduced sum divided by the worker count inside the library."""
         g = grad.reshape(-1).clone()
         if dist.get_backend(self.group) == "nccl":
             dist.all_reduce(g, op=dist.ReduceOp.SUM, group=self.group)
@@ -83,8 +91,7 @@ class DistributedA2SGD:
             h = g.cpu()
             dist.all_reduce(h, op=dist.ReduceOp.SUM, group=self.group)
             g.copy_(h)
-        # the sum over ranks enters the kernel; its 1/W factor rides on the learning rate
-        B.a2sgd_dense_sync(self.local, w, g.view(1, -1), lr / self.world)
+        B.a2sgd_dense_sync_reduced(self.local, w, g, self.world, lr)
 
     def destroy(self) -> None:
         self.local.destroy()

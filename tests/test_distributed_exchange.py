@@ -44,8 +44,8 @@ CPU_WORKER = textwrap.dedent("""
     lm = torch.tensor([[1.0 + rank, 10.0 * (rank + 1)]])
     gathered = D.exchange_local_means(lm)
     assert gathered.tolist() == [[1.0, 10.0], [2.0, 20.0]], gathered
-    avg = D.average_local_means(lm)
-    assert avg.tolist() == [1.5, 15.0], avg
+    sums = D.sum_local_means(lm)
+    assert sums.dtype == torch.float64 and sums.tolist() == [3.0, 30.0], sums
     dist.barrier()
     dist.destroy_process_group()
     print("rank", rank, "ok")

@@ -78,3 +78,69 @@ def test_reference_arm_json_line_has_the_contract_keys():
     assert line["impl"] == "reference" and line["cpu_baseline"]["kind"] == "oracle" and line["cpu_baseline"]["cores"] == 1
     assert line["e2e"]["h2d_bytes_per_step"] == 0 and line["e2e"]["d2h_bytes_per_step"] == 0
     assert line["value"] > 0 and line["config"]["workload"] == "c1_flat_1m"
+
+
+EXCHANGE_WORKER = textwrap.dedent("""
+    import os, sys
+    sys.path.insert(0, {root!r})
+    import torch
+    import torch.distributed as dist
+    import bench
+    from paper_2006_07405_b200 import distributed as D
+    dist.init_process_group("gloo", init_method="tcp://127.0.0.1:{port}", rank=int(sys.argv[1]), world_size=2)
+    rank = dist.get_rank()
+
+    class FakeWorker:
+        # the exchange itself is real (gloo); the kernels around it are not needed for the protocol
+        def __init__(self, exchange):
+            self.exchange, self.calls, self.destroyed = exchange, 0, False
+            self.local_means = torch.tensor([[1.0 + rank, 2.0 + rank]])
+        def exchange_means(self):
+            self.calls += 1
+            if self.exchange == "allgather":
+                got = D.exchange_local_means(self.local_means)
+                assert got.tolist() == [[1.0, 2.0], [2.0, 3.0]]
+            else:
+                assert D.sum_local_means(self.local_means).tolist() == [3.0, 5.0]
+        def destroy(self):
+            self.destroyed = True
+
+    made = []
+    def make_case(n, exchange):
+        w = FakeWorker(exchange)
+        made.append(w)
+        return w, w.exchange_means
+    out = bench.exchange_leg([1000, 2000], make_case, dist, torch.device("cpu"), steps=4, warmup=1,
+                             timer=bench.HostTimer())
+    assert out["workers"] == 2 and out["payload_bytes_per_worker"] == 8
+    assert sorted(out["sizes"]) == ["1000", "2000"]
+    for n, row in out["sizes"].items():
+        for ex in ("allgather", "allreduce"):
+            r = row[ex]
+            assert r["ms_per_step"] > 0 and r["us_per_exchange"] > 0
+            assert abs(r["worker_params_per_s"] - 2 * int(n) / (r["ms_per_step"] * 1e-3)) < 1e-3 * r["worker_params_per_s"]
+    assert len(made) == 4 and all(w.destroyed for w in made)
+    # warm-up 3 + 4 timed steps, then warm-up 3 + 50 timed exchanges
+    assert all(w.calls == 3 + 4 + 3 + 50 for w in made), [w.calls for w in made]
+    # both ranks hold the same (max over ranks) figures
+    flat = torch.tensor([out["sizes"][n][ex][k] for n in sorted(out["sizes"]) for ex in ("allgather", "allreduce")
+                         for k in ("ms_per_step", "us_per_exchange")], dtype=torch.float64)
+    other = [torch.zeros_like(flat) for _ in range(2)]
+    dist.all_gather(other, flat)
+    assert torch.equal(other[0], other[1])
+    dist.barrier()
+    dist.destroy_process_group()
+    print("rank", rank, "ok")
+""")
+
+
+def test_exchange_leg_protocol_world_size_2(tmp_path):
+    port = _free_port()
+    script = tmp_path / "worker.py"
+    script.write_text(EXCHANGE_WORKER.format(root=ROOT, port=port))
+    procs = [subprocess.Popen([sys.executable, str(script), str(r)], stdout=subprocess.PIPE,
+                              stderr=subprocess.STDOUT, text=True) for r in range(2)]
+    outs = [p.communicate(timeout=180)[0] for p in procs]
+    for r, (p, out) in enumerate(zip(procs, outs)):
+        assert p.returncode == 0, out
+        assert f"rank {r} ok" in out
