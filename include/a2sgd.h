@@ -71,7 +71,8 @@ enum a2sgd_status {
     A2SGD_ERR_TIMEOUT = -4,   /* a bounded device-side wait ran out (latched in the status word) */
     A2SGD_ERR_NONFINITE = -5, /* a group sum was NaN or Inf (latched in the status word) */
     A2SGD_ERR_NOMEM = -6,     /* scratch allocation failed */
-    A2SGD_ERR_TOO_LARGE = -7  /* n*P exceeds what the single-launch path can hold on chip */
+    A2SGD_ERR_TOO_LARGE = -7  /* n*P exceeds what the single-launch path can hold on chip (A2SGD_FORCE_COOPERATIVE),
+                                 or P > A2SGD_NOALLOC_MAX_P in a2sgd_encode_noalloc (its fixed scratch) */
 };
 
 enum a2sgd_flags {

@@ -1176,7 +1176,7 @@ extern "C" const char *a2sgd_status_string(int status)
     case A2SGD_ERR_TIMEOUT: return "bounded device-side wait ran out";
     case A2SGD_ERR_NONFINITE: return "non-finite group sum";
     case A2SGD_ERR_NOMEM: return "scratch allocation failed";
-    case A2SGD_ERR_TOO_LARGE: return "n*P too large for the single-launch path";
+    case A2SGD_ERR_TOO_LARGE: return "too large: n*P for the single-launch path, or P for the fixed scratch";
     default: return "unknown status";
     }
 }

@@ -12,6 +12,7 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
 from paper_2006_07405_b200 import binding as B
 from parity_util import assert_means
 
@@ -44,7 +45,31 @@ def test_noalloc_encode_matches_regular_encode_twice(mode, P, n, stride):
         assert torch.equal(cnt, cnt_ref)                                   # integers: equal
         assert_means(lm_buf[1:P + 1].cpu().numpy(), lm_ref.cpu().numpy())   # 1e-6, as everywhere
         assert torch.isnan(lm_buf[0]).all() and torch.isnan(lm_buf[P + 1]).all()
+        # and directly against the CPU oracle on the same inputs
+        lm_o, cnt_o, _ = oracle.encode(g.cpu().numpy(), e.cpu().numpy() if mode == B.MODE_EF else None, mode=mode)
+        assert np.array_equal(cnt.cpu().numpy().astype(np.uint64), cnt_o)
+        assert_means(lm_buf[1:P + 1].cpu().numpy(), lm_o)
     ctx.destroy()
+
+
+def test_noalloc_calls_leave_device_memory_as_it_was():
+    """What the entry point exists for: after a first call has done its one-time set-up, further
+    calls neither take nor return device memory — seen from the driver (free bytes) and from the
+    caller's own allocator."""
+    P, n = 4, 1 << 20
+    g, e = _inputs(7, P, n, n)
+    lm = torch.zeros((P, 2), device="cuda")
+    cnt = torch.zeros(P, dtype=torch.int64, device="cuda")
+    B.a2sgd_encode_noalloc(g, e, lm, cnt)          # first call on this device: symbol look-up, module load
+    torch.cuda.synchronize()
+    free_before, _ = torch.cuda.mem_get_info()
+    held_before = torch.cuda.memory_allocated()
+    for _ in range(2):
+        B.a2sgd_encode_noalloc(g, e, lm, cnt)
+    torch.cuda.synchronize()
+    free_after, _ = torch.cuda.mem_get_info()
+    assert free_after == free_before
+    assert torch.cuda.memory_allocated() == held_before
 
 
 def test_noalloc_rejects_what_the_fixed_scratch_cannot_hold():
