@@ -286,17 +286,24 @@ def host_description() -> dict:
     return {"nproc": os.cpu_count(), "usable_cores": usable, "cpu_model": model}
 
 
-def time_workload(wl, steps, warmup, dev, *, with_roofline=True, with_next_rows=True, with_e2e=True, dist=None):
-    """Runs the timed regions for one workload on this rank's GPU.  Returns a dict of results."""
+def time_workload(wl, steps, warmup, dev, *, with_roofline=True, with_next_rows=True, with_e2e=True, dist=None,
+                  row_stride=None):
+    """Runs the timed regions for one workload on this rank's GPU.  Returns a dict of results.
+    ``row_stride`` overrides the 128-byte aligned row layout (e.g. n + 1: every row at a different
+    4-byte phase, which takes the general-alignment kernels)."""
     import torch
     from paper_2006_07405_b200 import binding as B
     from paper_2006_07405_b200 import workloads as W
 
     n, P = wl.n, wl.P
     torch.cuda.set_device(dev)
-    # rows start 128-byte aligned (row stride = n rounded up to 32 elements)
-    g = B.padded_rows(P, n, dev)
-    e = B.padded_rows(P, n, dev, fill=0.0)
+    if row_stride is None:
+        # rows start 128-byte aligned (row stride = n rounded up to 32 elements)
+        g = B.padded_rows(P, n, dev)
+        e = B.padded_rows(P, n, dev, fill=0.0)
+    else:
+        g = torch.empty((P, row_stride), device=dev)[:, :n]
+        e = torch.zeros((P, row_stride), device=dev)[:, :n]
     w = torch.empty(n, device=dev)
     W.fill_gradients(wl, 0, g)
     W.init_weights(wl, w)
@@ -741,6 +748,10 @@ def main():
             k = 20 if w2.n > 10 ** 9 else (100 if w2.n > 10 ** 7 else 1000)
             r2 = time_workload(w2, k, 3, dev, with_e2e=False)
             extra[name] = summarise(w2, r2, 1, peak_gbs)
+        # rows that are only 4-byte aligned, each at a different phase: the general-alignment kernels
+        w2 = W.get_workload(FALLBACK_WORKLOAD)
+        r2 = time_workload(w2, 100, 3, dev, with_e2e=False, with_next_rows=False, row_stride=w2.n + 1)
+        extra[f"{w2.name}, rows misaligned (row stride n + 1, 32-bit coalesced accesses)"] = summarise(w2, r2, 1, peak_gbs)
 
     exchange = None
     if dist is not None and ((world > 1 and not args.no_extra) or args.exchange_leg):

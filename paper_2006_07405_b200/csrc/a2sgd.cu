@@ -398,7 +398,7 @@ int launch_encode(a2sgd_ctx *c, const float *grad, int64_t gs, const float *err,
     const int vw = encode_vec_width(c, grad, gs, err, es);
     EncodeArgs a = make_encode_args(c, grad, gs, err, es, local_means, pos_counts, pos_mask, global_means);
     const void *fn = select_encode(!c->alg1, pos_mask != nullptr, vw);
-    const uint64_t items = vw ? (c->n + vw - 1) / vw : c->n;
+    const uint64_t items = vw ? (c->n + vw - 1) / vw : (c->n + kScalarU - 1) / kScalarU;
     const dim3 grid(std::min(per_worker_grid(c, occupancy(c, fn), items, A2SGD_WAVES_K1), c->g_alloc), c->P);
     void *params[] = {&a};
     A2_CUDA(launch_pdl(fn, grid, params, s));
@@ -441,8 +441,9 @@ int launch_decode(a2sgd_ctx *c, float *w, int64_t ws, const float *grad, int64_t
         grid = dim3(per_worker_grid(c, occupancy(c, fn), (c->n + vw - 1) / vw, A2SGD_WAVES_K3), c->P);
     } else {
         fn = select_decode_scalar(ef, store, mom);
-        grid = shared ? dim3(flat_grid(c, occupancy(c, fn), c->n, A2SGD_WAVES_K3), 1)
-                      : dim3(per_worker_grid(c, occupancy(c, fn), c->n, A2SGD_WAVES_K3), c->P);
+        const uint64_t items = (c->n + kDecScalarU - 1) / kDecScalarU; // one tile of kBlock * kDecScalarU per CTA
+        grid = shared ? dim3(flat_grid(c, occupancy(c, fn), items, A2SGD_WAVES_K3), 1)
+                      : dim3(per_worker_grid(c, occupancy(c, fn), items, A2SGD_WAVES_K3), c->P);
     }
     A2_CUDA(launch_pdl(fn, grid, params, s));
     return A2SGD_OK;
@@ -862,7 +863,7 @@ static int step_lowp(a2sgd_ctx *c, float *w, int64_t w_stride, const uint16_t *g
         EncodeArgs a = make_encode_args(c, g, grad_stride, err, err_stride, c->local_means, c->pos_counts, nullptr,
                                         c->global_means);
         const void *fn = gt == 1 ? select_encode_lowp<1>(ef, vw_enc) : select_encode_lowp<2>(ef, vw_enc);
-        const uint64_t items = vw_enc ? (c->n + 7) / 8 : c->n;
+        const uint64_t items = vw_enc ? (c->n + 7) / 8 : (c->n + kScalarU - 1) / kScalarU;
         const dim3 grid(std::min(per_worker_grid(c, occupancy(c, fn), items, A2SGD_WAVES_K1), c->g_alloc), c->P);
         void *params[] = {&a};
         A2_CUDA(launch_pdl(fn, grid, params, s));
@@ -871,7 +872,7 @@ static int step_lowp(a2sgd_ctx *c, float *w, int64_t w_stride, const uint16_t *g
         DecodeArgs a = make_decode_args(c, w, ws, g, grad_stride, err, err_stride, c->local_means, c->global_means, lr);
         const void *fn = gt == 1 ? select_decode_lowp<1>(ef, store, ws == 0, c->P, vw_dec)
                                  : select_decode_lowp<2>(ef, store, ws == 0, c->P, vw_dec);
-        const uint64_t items = vw_dec ? (c->n + 7) / 8 : c->n;
+        const uint64_t items = vw_dec ? (c->n + 7) / 8 : (c->n + kDecScalarU - 1) / kDecScalarU;
         const dim3 grid = (ws == 0) ? dim3(flat_grid(c, occupancy(c, fn), items, A2SGD_WAVES_K3))
                                     : dim3(per_worker_grid(c, occupancy(c, fn), items, A2SGD_WAVES_K3), c->P);
         void *params[] = {&a};

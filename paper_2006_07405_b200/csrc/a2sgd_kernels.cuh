@@ -506,7 +506,14 @@ __global__ void __launch_bounds__(kBlock) k_encode_vec(EncodeArgs a)
     finish_worker(a, p, s_pos, s_neg, n_pos, sh_d, sh_n, &sh_flag);
 }
 
-// General path: any 4-byte alignment, scalar coalesced accesses.  grid = (G, P).
+// General path: any 4-byte alignment, coalesced 32-bit accesses.  grid = (G, P).
+// A CTA walks tiles of kBlock * kScalarU consecutive elements; within a tile a thread takes the
+// elements tid, tid + kBlock, ... so that every load instruction of a warp is one contiguous
+// 128-byte piece whatever the row's alignment.  All loads of a tile are issued before the first
+// use, the kScalarU values are summed pairwise in fp32 and enter the fp64 running sums once per
+// tile — the same arithmetic shape as the vector kernel, only with narrower accesses.
+constexpr int kScalarU = 8;
+
 template <bool EF, bool MASK, int GB = 0>
 __global__ void __launch_bounds__(kBlock) k_encode_scalar(EncodeArgs a)
 {
@@ -522,22 +529,43 @@ __global__ void __launch_bounds__(kBlock) k_encode_scalar(EncodeArgs a)
     const float *__restrict__ e = EF ? a.err + (int64_t)p * a.err_stride : nullptr;
     uint32_t *mask = MASK ? a.pos_mask + (uint64_t)p * ((a.n + 31) >> 5) : nullptr;
     const unsigned lane = threadIdx.x & 31u;
-    const uint64_t stride = (uint64_t)gridDim.x * kBlock;
+    constexpr uint64_t kTile = (uint64_t)kBlock * kScalarU;
+    const uint64_t tiles = (a.n + kTile - 1) / kTile;
     Acc acc;
-    for (uint64_t i = (uint64_t)blockIdx.x * kBlock + threadIdx.x; (i - lane) < a.n; i += stride) {
-        float sp = 0.f, sn = 0.f;
-        unsigned bit = 0;
-        if (i < a.n) {
-            float v = g.one(i);
-            if (EF) v += ld_stream1(e + i);
-            split1(v, sp, sn, acc.n_pos, bit);
+    for (uint64_t t = blockIdx.x; t < tiles; t += gridDim.x) {
+        const uint64_t base = t * kTile + threadIdx.x;
+        float gv[kScalarU], ev[kScalarU];
+        const bool whole = (t + 1) * kTile <= a.n;
+        if (whole) {
+#pragma unroll
+            for (int k = 0; k < kScalarU; ++k) gv[k] = g.one(base + (uint64_t)k * kBlock);
+            if (EF) {
+#pragma unroll
+                for (int k = 0; k < kScalarU; ++k) ev[k] = ld_stream1(e + base + (uint64_t)k * kBlock);
+            }
+        } else {
+#pragma unroll
+            for (int k = 0; k < kScalarU; ++k) {
+                const uint64_t i = base + (uint64_t)k * kBlock;
+                gv[k] = i < a.n ? g.one(i) : 0.f;
+                ev[k] = (EF && i < a.n) ? ld_stream1(e + i) : 0.f;
+            }
         }
-        acc.s_pos += (double)sp;
-        acc.s_neg += (double)sn;
-        if (MASK) {
-            const unsigned w = __ballot_sync(0xffffffffu, bit != 0);
-            if (lane == 0) mask[i >> 5] = w;
+        float sp[kScalarU], sn[kScalarU];
+#pragma unroll
+        for (int k = 0; k < kScalarU; ++k) {
+            const uint64_t i = base + (uint64_t)k * kBlock;
+            const float v = EF ? gv[k] + ev[k] : gv[k];
+            unsigned bit = 0;
+            sp[k] = sn[k] = 0.f;
+            if (whole || i < a.n) split1(v, sp[k], sn[k], acc.n_pos, bit);
+            if (MASK && (whole || (i - lane) < a.n)) {       // warp-uniform: the warp's 32 elements share a word
+                const unsigned w = __ballot_sync(0xffffffffu, bit != 0);
+                if (lane == 0) mask[i >> 5] = w;
+            }
         }
+        acc.s_pos += (double)tree_sum<kScalarU>(sp);
+        acc.s_neg += (double)tree_sum<kScalarU>(sn);
     }
     double s_pos = acc.s_pos, s_neg = acc.s_neg;
     unsigned long long n_pos = acc.n_pos;
@@ -871,35 +899,86 @@ __global__ void __launch_bounds__(kBlock) k_decode_repl_vec(DecodeArgs a)
     }
 }
 
-// General path: any 4-byte alignment, both weight layouts, scalar accesses.
-// Shared w: grid = (G, 1), the thread walks the workers; replicas: grid = (G, P).
+// General path: any 4-byte alignment, both weight layouts, coalesced 32-bit accesses.
+// One tile of kBlock * kDecScalarU consecutive model elements per CTA (grid.x = number of tiles);
+// a thread takes the elements tid, tid + kBlock, ... of the tile.  Shared w: grid = (tiles, 1), the
+// thread walks the workers in batches of four with all loads of a batch issued before its first
+// store; replicas: grid = (tiles, P).
+constexpr int kDecScalarU = 4;
+
 template <bool EF, bool STORE, int GB = 0, bool MOM = false>
 __global__ void __launch_bounds__(kBlock) k_decode_scalar(DecodeArgs a)
 {
     pdl_wait_prior_grid();
     pdl_release_next_grid();
 
+    __shared__ WorkerConst sh_c[kMaxP];
     const float m_pos = __ldg(a.global_means), m_neg = __ldg(a.global_means + 1);
-    const uint64_t stride = (uint64_t)gridDim.x * kBlock;
     const bool shared = a.w_stride == 0;
     const uint32_t p_lo = shared ? 0 : blockIdx.y, p_hi = shared ? a.P : blockIdx.y + 1;
     const UpdateConst uc = update_const(a, shared ? (float)a.P : 1.0f);
-    for (uint64_t i = (uint64_t)blockIdx.x * kBlock + threadIdx.x; i < a.n; i += stride) {
-        float sum = 0.f;
-        for (uint32_t p = p_lo; p < p_hi; ++p) {
-            const WorkerConst c = worker_const<EF>(a, p, m_pos, m_neg);
-            float v = GradRow<GB>(a.grad, (int64_t)p * a.grad_stride).one(i);
-            if (EF) v += ld_stream1(a.err + (int64_t)p * a.err_stride + i);
-            float gh, rs;
-            decode1<EF>(v, c, gh, rs);
-            sum += gh;
-            if (STORE) st_stream1(a.err + (int64_t)p * a.err_stride + i, rs);
+    for (uint32_t p = p_lo + threadIdx.x; p < p_hi; p += kBlock) sh_c[p] = worker_const<EF>(a, p, m_pos, m_neg);
+    __syncthreads();
+
+    constexpr int U = kDecScalarU, PB = 4;
+    constexpr uint64_t kTile = (uint64_t)kBlock * U;
+    const uint64_t tiles = (a.n + kTile - 1) / kTile;
+    for (uint64_t t = blockIdx.x; t < tiles; t += gridDim.x) {
+        const uint64_t base = t * kTile + threadIdx.x;
+        bool live[U];
+        float wv[U], mv[U], sum[U];
+        float *wrow = a.w + (int64_t)p_lo * a.w_stride;
+        float *mrow = MOM ? a.mom + (int64_t)p_lo * a.mom_stride : nullptr;
+#pragma unroll
+        for (int k = 0; k < U; ++k) {
+            const uint64_t i = base + (uint64_t)k * kBlock;
+            live[k] = i < a.n;
+            wv[k] = live[k] ? ld_stream1(wrow + i) : 0.f;
+            mv[k] = (MOM && live[k]) ? ld_stream1(mrow + i) : 0.f;
+            sum[k] = 0.f;
         }
-        float *wp = a.w + (int64_t)p_lo * a.w_stride + i;
-        float *mp = MOM ? a.mom + (int64_t)p_lo * a.mom_stride + i : nullptr;
-        float m = MOM ? *mp : 0.f;
-        *wp = update1<MOM>(uc, sum, *wp, m);
-        if (MOM) *mp = m;
+        for (uint32_t p0 = p_lo; p0 < p_hi; p0 += PB) {
+            float gv[PB][U], ev[PB][U];
+#pragma unroll
+            for (int q = 0; q < PB; ++q) {
+                const bool wq = p0 + q < p_hi;
+                const GradRow<GB> g(a.grad, (int64_t)(wq ? p0 + q : p0) * a.grad_stride);
+#pragma unroll
+                for (int k = 0; k < U; ++k) gv[q][k] = (wq && live[k]) ? g.one(base + (uint64_t)k * kBlock) : 0.f;
+            }
+            if (EF) {
+#pragma unroll
+                for (int q = 0; q < PB; ++q) {
+                    const bool wq = p0 + q < p_hi;
+                    const float *e = a.err + (int64_t)(wq ? p0 + q : p0) * a.err_stride;
+#pragma unroll
+                    for (int k = 0; k < U; ++k) ev[q][k] = (wq && live[k]) ? ld_stream1(e + base + (uint64_t)k * kBlock) : 0.f;
+                }
+            }
+#pragma unroll
+            for (int q = 0; q < PB; ++q) {
+                if (p0 + q >= p_hi) break;
+                const WorkerConst c = sh_c[p0 + q];
+                float *e = STORE ? a.err + (int64_t)(p0 + q) * a.err_stride : nullptr;
+#pragma unroll
+                for (int k = 0; k < U; ++k) {
+                    if (!live[k]) continue;
+                    const float v = EF ? gv[q][k] + ev[q][k] : gv[q][k];
+                    float gh, rs;
+                    decode1<EF>(v, c, gh, rs);
+                    sum[k] += gh;
+                    if (STORE) st_stream1(e + base + (uint64_t)k * kBlock, rs);
+                }
+            }
+        }
+#pragma unroll
+        for (int k = 0; k < U; ++k) {
+            if (!live[k]) continue;
+            const uint64_t i = base + (uint64_t)k * kBlock;
+            float m = mv[k];
+            st_stream1(wrow + i, update1<MOM>(uc, sum[k], wv[k], m));
+            if (MOM) st_stream1(mrow + i, m);
+        }
     }
 }
 

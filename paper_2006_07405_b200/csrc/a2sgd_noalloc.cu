@@ -130,7 +130,7 @@ extern "C" int a2sgd_encode_noalloc(uint64_t n, uint32_t P, uint32_t mode, const
         (void)cudaGetLastError();
         occ = 1;
     }
-    const uint64_t items = vw ? (n + vw - 1) / vw : n;
+    const uint64_t items = vw ? (n + vw - 1) / vw : (n + kScalarU - 1) / kScalarU;
     const uint64_t slots = (uint64_t)setup->sm_count * (uint64_t)std::max(occ, 1);
     uint64_t G = std::max<uint64_t>(1, std::min<uint64_t>(slots, kNoAllocMaxCtas) / P);
     G = std::min<uint64_t>(G, std::max<uint64_t>(1, (items + kBlock - 1) / kBlock));
