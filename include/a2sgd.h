@@ -261,6 +261,17 @@ int a2sgd_step_segments(a2sgd_ctx *ctx, a2sgd_segments *plan, float lr, void *st
  * paper's experimental setup for VGG-16); computing those rates is the caller's business. */
 int a2sgd_step_segments_lr(a2sgd_ctx *ctx, a2sgd_segments *plan, const float *lr_per_segment, void *stream);
 
+/* The two stages of a2sgd_step_segments as separate calls, mirroring a2sgd_encode and
+ * a2sgd_decode_update (Algorithm 1 line 3, and lines 4, 6, 7) for a segment list; the 2P scalars
+ * are averaged in between with a2sgd_global_average (line 5).
+ *   local_means   DEVICE [P][2] (out of the first call, in of the second: read in ALG1 mode only)
+ *   pos_counts    DEVICE [P], may be NULL;   global_means  DEVICE [2]
+ *   lr_per_segment  DEVICE [S] or NULL (then `lr` applies to every tensor) */
+int a2sgd_encode_segments(a2sgd_ctx *ctx, a2sgd_segments *plan, float *local_means, uint64_t *pos_counts,
+                          void *stream);
+int a2sgd_decode_update_segments(a2sgd_ctx *ctx, a2sgd_segments *plan, const float *local_means,
+                                 const float *global_means, float lr, const float *lr_per_segment, void *stream);
+
 /* a2sgd_step for a caller whose fresh gradients sit in HOST memory (pinned
  * memory makes the copies asynchronous): copies grad_host -> grad_staging
  * worker by worker, runs the step, copies the 2P local and 2 global means

@@ -90,6 +90,10 @@ def lib() -> ctypes.CDLL:
                                             ctypes.c_int, ctypes.POINTER(_vp)]
         l.a2sgd_segments_destroy.restype = ctypes.c_int
         l.a2sgd_segments_destroy.argtypes = [_vp]
+        l.a2sgd_encode_segments.restype = ctypes.c_int
+        l.a2sgd_encode_segments.argtypes = [_vp, _vp, _vp, _vp, _vp]
+        l.a2sgd_decode_update_segments.restype = ctypes.c_int
+        l.a2sgd_decode_update_segments.argtypes = [_vp, _vp, _vp, _vp, ctypes.c_float, _vp, _vp]
         l.a2sgd_step_segments.restype = ctypes.c_int
         l.a2sgd_step_segments.argtypes = [_vp, _vp, ctypes.c_float, _vp]
         for fn in (l.a2sgd_step_bf16, l.a2sgd_step_f16):
@@ -373,6 +377,23 @@ def a2sgd_segments_destroy(plan: Segments) -> None:
 
 def a2sgd_step_segments(ctx: Context, plan: Segments, lr: float, stream=None) -> None:
     _check(lib().a2sgd_step_segments(ctx.handle, plan.handle, float(lr), _stream(stream)), "a2sgd_step_segments")
+
+
+def a2sgd_encode_segments(ctx: Context, plan: Segments, local_means: torch.Tensor,
+                          pos_counts: Optional[torch.Tensor] = None, stream=None) -> None:
+    _check(lib().a2sgd_encode_segments(ctx.handle, plan.handle, local_means.data_ptr(),
+                                       pos_counts.data_ptr() if pos_counts is not None else None, _stream(stream)),
+           "a2sgd_encode_segments")
+
+
+def a2sgd_decode_update_segments(ctx: Context, plan: Segments, local_means: Optional[torch.Tensor],
+                                 global_means: torch.Tensor, lr: float,
+                                 lr_per_segment: Optional[torch.Tensor] = None, stream=None) -> None:
+    _check(lib().a2sgd_decode_update_segments(ctx.handle, plan.handle,
+                                              local_means.data_ptr() if local_means is not None else None,
+                                              global_means.data_ptr(), float(lr),
+                                              lr_per_segment.data_ptr() if lr_per_segment is not None else None,
+                                              _stream(stream)), "a2sgd_decode_update_segments")
 
 
 def a2sgd_step_segments_lr(ctx: Context, plan: Segments, lr_per_segment: torch.Tensor, stream=None) -> None:

@@ -15,27 +15,21 @@
 
 using namespace a2sgd;
 
-// Grid shapes (measured on B200, CUDA events, c2/c3/c4 workloads):
+// Grid shapes (measured on B200, CUDA events, c2-c5 workloads):
 //  * decode: one vector per thread, as many CTAs as that takes.  A persistent grid of
 //    148 x occupancy CTAs with an equal static share each ran the same kernel at 6.2 TB/s; the
 //    SMs do not stream at equal speed (two dies, shared channels), so the slowest share set the
 //    time.  Letting the hardware CTA scheduler hand out small CTAs reaches 6.9-7.0 TB/s.
 //  * encode: per-CTA partial sums must stay few and their order fixed, so the grid stays
-//    proportional to the resident-CTA count; two CTAs per resident slot is the best measured.
-#ifndef A2SGD_WAVES_K1
-#define A2SGD_WAVES_K1 2
-#endif
-#ifndef A2SGD_WAVES_K1_DEFERRED
-#define A2SGD_WAVES_K1_DEFERRED 16 /* the deferred-residual encode also writes v: a read/write mix, and like the
-                                      decode kernels it gains from many CTAs per slot (c2: 626 us per step at 1,
-                                      602 at 4, 583 at 16 and 32, 599 at 64) */
-#endif
-#ifndef A2SGD_WAVES_K3
-#define A2SGD_WAVES_K3 (1 << 20) /* effectively: cover every vector with its own thread */
-#endif
-#ifndef A2SGD_MAX_VW
-#define A2SGD_MAX_VW 8 /* widest vector access the dispatcher may pick: 8 = 256-bit, 4 = 128-bit */
-#endif
+//    proportional to the resident-CTA count: 16 CTAs per resident slot (1 -> 2 -> 4 -> 16 measured
+//    7.18 -> 7.27 -> 7.33 -> 7.36 TB/s on c5 and 7.02 -> 7.13 -> 7.18 -> 7.24 on c4; the fold of
+//    the 18944 / P partials per worker by the last CTA stays negligible).  The deferred-residual
+//    encode also writes v, a read/write mix, and gains the same way (c2: 626 us per step at 1,
+//    583 at 16 and 32, 599 at 64).
+constexpr int kWavesK1 = 16;
+constexpr int kWavesK1Deferred = 16;
+constexpr int kWavesK3 = 1 << 20; // effectively: cover every vector with its own thread
+constexpr int kMaxVecWidth = 8;   // widest access the dispatcher picks: 256-bit
 
 struct a2sgd_ctx {
     uint64_t n = 0;
@@ -70,6 +64,7 @@ struct a2sgd_segments {
     bool has_err = false;
     // device tables
     SegTile *tiles = nullptr;
+    SegStart *starts = nullptr; // [S + 1], only for S <= kSegScanMax
     uint64_t n_tiles = 0;
     uint64_t *numel = nullptr;
     const float **grad = nullptr;
@@ -114,14 +109,10 @@ inline bool stride_ok(int64_t stride, uint64_t n, uint32_t P)
 inline int vec_width(const void *p, int64_t stride, uint32_t P)
 {
     if (p == nullptr) return 8;
-    if (A2SGD_MAX_VW >= 8 && aligned(p, 32) && (P == 1 || stride % 8 == 0)) return 8;
+    if (kMaxVecWidth >= 8 && aligned(p, 32) && (P == 1 || stride % 8 == 0)) return 8;
     if (aligned(p, 16) && (P == 1 || stride % 4 == 0)) return 4;
     return 0;
 }
-
-#ifndef A2SGD_PDL
-#define A2SGD_PDL 1
-#endif
 
 // Launch with programmatic stream serialisation (see pdl_wait_prior_grid in the kernels).
 cudaError_t launch_pdl(const void *fn, dim3 grid, void **params, cudaStream_t s)
@@ -133,7 +124,7 @@ cudaError_t launch_pdl(const void *fn, dim3 grid, void **params, cudaStream_t s)
     cfg.stream = s;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = A2SGD_PDL;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     return cudaLaunchKernelExC(&cfg, fn, params);
@@ -399,7 +390,7 @@ int launch_encode(a2sgd_ctx *c, const float *grad, int64_t gs, const float *err,
     EncodeArgs a = make_encode_args(c, grad, gs, err, es, local_means, pos_counts, pos_mask, global_means);
     const void *fn = select_encode(!c->alg1, pos_mask != nullptr, vw);
     const uint64_t items = vw ? (c->n + vw - 1) / vw : (c->n + kScalarU - 1) / kScalarU;
-    const dim3 grid(std::min(per_worker_grid(c, occupancy(c, fn), items, A2SGD_WAVES_K1), c->g_alloc), c->P);
+    const dim3 grid(std::min(per_worker_grid(c, occupancy(c, fn), items, kWavesK1), c->g_alloc), c->P);
     void *params[] = {&a};
     A2_CUDA(launch_pdl(fn, grid, params, s));
     return A2SGD_OK;
@@ -435,15 +426,15 @@ int launch_decode(a2sgd_ctx *c, float *w, int64_t ws, const float *grad, int64_t
     dim3 grid;
     if (vw && shared) {
         fn = select_decode_shared(ef, store, c->P, vw, mom);
-        grid = dim3(flat_grid(c, occupancy(c, fn), (c->n + vw - 1) / vw, A2SGD_WAVES_K3));
+        grid = dim3(flat_grid(c, occupancy(c, fn), (c->n + vw - 1) / vw, kWavesK3));
     } else if (vw) {
         fn = select_decode_repl(ef, store, vw, mom);
-        grid = dim3(per_worker_grid(c, occupancy(c, fn), (c->n + vw - 1) / vw, A2SGD_WAVES_K3), c->P);
+        grid = dim3(per_worker_grid(c, occupancy(c, fn), (c->n + vw - 1) / vw, kWavesK3), c->P);
     } else {
         fn = select_decode_scalar(ef, store, mom);
         const uint64_t items = (c->n + kDecScalarU - 1) / kDecScalarU; // one tile of kBlock * kDecScalarU per CTA
-        grid = shared ? dim3(flat_grid(c, occupancy(c, fn), items, A2SGD_WAVES_K3), 1)
-                      : dim3(per_worker_grid(c, occupancy(c, fn), items, A2SGD_WAVES_K3), c->P);
+        grid = shared ? dim3(flat_grid(c, occupancy(c, fn), items, kWavesK3), 1)
+                      : dim3(per_worker_grid(c, occupancy(c, fn), items, kWavesK3), c->P);
     }
     A2_CUDA(launch_pdl(fn, grid, params, s));
     return A2SGD_OK;
@@ -529,7 +520,7 @@ int deferred_step(a2sgd_ctx *c, float *w, int64_t ws, const float *grad, int64_t
         a.prev_means = c->prev_means;
         const void *fn = c->err_holds_v ? (const void *)k_encode_vec<true, true, 8, false, 2>
                                         : (const void *)k_encode_vec<true, true, 8, false, 1>;
-        const dim3 grid(std::min(per_worker_grid(c, occupancy(c, fn), (c->n + 7) / 8, A2SGD_WAVES_K1_DEFERRED), c->g_alloc), c->P);
+        const dim3 grid(std::min(per_worker_grid(c, occupancy(c, fn), (c->n + 7) / 8, kWavesK1Deferred), c->g_alloc), c->P);
         void *params[] = {&a};
         A2_CUDA(launch_pdl(fn, grid, params, s));
     }
@@ -546,7 +537,7 @@ int deferred_step(a2sgd_ctx *c, float *w, int64_t ws, const float *grad, int64_t
         a.prev_means = c->prev_means;
         a.lr = lr;
         const void *fn = ws == 0 ? select_decode_deferred<false>(c->P) : select_decode_deferred<true>(c->P);
-        const dim3 grid(flat_grid(c, occupancy(c, fn), std::max<uint64_t>(1, (c->n / 32) * 4), A2SGD_WAVES_K3));
+        const dim3 grid(flat_grid(c, occupancy(c, fn), std::max<uint64_t>(1, (c->n / 32) * 4), kWavesK3));
         void *params[] = {&a};
         A2_CUDA(launch_pdl(fn, grid, params, s));
     }
@@ -617,7 +608,7 @@ extern "C" int a2sgd_create(a2sgd_ctx **out, uint64_t n, uint32_t P, int device,
         c->l2_bytes = (size_t)std::max(l2, 0);
     }
     // partials: room for a (G, P) grid that fills the device at the highest possible occupancy
-    const uint32_t max_slots = (uint32_t)c->sm_count * (2048 / kBlock) * std::max(A2SGD_WAVES_K1, A2SGD_WAVES_K1_DEFERRED);
+    const uint32_t max_slots = (uint32_t)c->sm_count * (2048 / kBlock) * std::max(kWavesK1, kWavesK1Deferred);
     c->g_alloc = std::max<uint32_t>(1, max_slots / P);
     bool ok = true;
     ok = ok && cudaMalloc(&c->partials, sizeof(Partial) * (size_t)c->g_alloc * P) == cudaSuccess;
@@ -864,7 +855,7 @@ static int step_lowp(a2sgd_ctx *c, float *w, int64_t w_stride, const uint16_t *g
                                         c->global_means);
         const void *fn = gt == 1 ? select_encode_lowp<1>(ef, vw_enc) : select_encode_lowp<2>(ef, vw_enc);
         const uint64_t items = vw_enc ? (c->n + 7) / 8 : (c->n + kScalarU - 1) / kScalarU;
-        const dim3 grid(std::min(per_worker_grid(c, occupancy(c, fn), items, A2SGD_WAVES_K1), c->g_alloc), c->P);
+        const dim3 grid(std::min(per_worker_grid(c, occupancy(c, fn), items, kWavesK1), c->g_alloc), c->P);
         void *params[] = {&a};
         A2_CUDA(launch_pdl(fn, grid, params, s));
     }
@@ -873,8 +864,8 @@ static int step_lowp(a2sgd_ctx *c, float *w, int64_t w_stride, const uint16_t *g
         const void *fn = gt == 1 ? select_decode_lowp<1>(ef, store, ws == 0, c->P, vw_dec)
                                  : select_decode_lowp<2>(ef, store, ws == 0, c->P, vw_dec);
         const uint64_t items = vw_dec ? (c->n + 7) / 8 : (c->n + kDecScalarU - 1) / kDecScalarU;
-        const dim3 grid = (ws == 0) ? dim3(flat_grid(c, occupancy(c, fn), items, A2SGD_WAVES_K3))
-                                    : dim3(per_worker_grid(c, occupancy(c, fn), items, A2SGD_WAVES_K3), c->P);
+        const dim3 grid = (ws == 0) ? dim3(flat_grid(c, occupancy(c, fn), items, kWavesK3))
+                                    : dim3(per_worker_grid(c, occupancy(c, fn), items, kWavesK3), c->P);
         void *params[] = {&a};
         A2_CUDA(launch_pdl(fn, grid, params, s));
     }
@@ -938,7 +929,7 @@ static int dense_sync_impl(a2sgd_ctx *c, float *w, int64_t w_stride, const float
     a.divisor = divisor;
     const void *fn = select_dense(c->P, vw, ws != 0);
     const uint64_t items = vw ? (c->n + vw - 1) / vw : c->n;
-    const dim3 grid(flat_grid(c, occupancy(c, fn), items, A2SGD_WAVES_K3));
+    const dim3 grid(flat_grid(c, occupancy(c, fn), items, kWavesK3));
     void *params[] = {&a};
     A2_CUDA(launch_pdl(fn, grid, params, static_cast<cudaStream_t>(stream)));
     return A2SGD_OK;
@@ -969,6 +960,7 @@ extern "C" int a2sgd_segments_create(a2sgd_ctx *c, uint32_t S, const uint64_t *n
     const bool repl = w_replicated != 0 && P > 1;
     uint64_t total = 0;
     std::vector<SegTile> tiles;
+    std::vector<SegStart> starts;
     for (uint32_t s = 0; s < S; ++s) {
         if (numel[s] == 0) return A2SGD_ERR_ARG;
         total += numel[s];
@@ -987,6 +979,7 @@ extern "C" int a2sgd_segments_create(a2sgd_ctx *c, uint32_t S, const uint64_t *n
             if (!aligned(wp, 4)) return A2SGD_ERR_ALIGN;
             vec = vec && aligned(wp, 32);
         }
+        starts.push_back(SegStart{(uint64_t)tiles.size(), numel[s], vec ? kSegFlagVec : 0u, {0u, 0u, 0u}});
         for (uint64_t off = 0; off < numel[s]; off += kSegTile) tiles.push_back(SegTile{s, vec ? kSegFlagVec : 0u, off});
     }
     if (total != c->n) return A2SGD_ERR_ARG;
@@ -1007,6 +1000,11 @@ extern "C" int a2sgd_segments_create(a2sgd_ctx *c, uint32_t S, const uint64_t *n
     ok = ok && cudaMalloc(&sg->w, sizeof(float *) * w_count) == cudaSuccess;
     if (err) ok = ok && cudaMalloc(&sg->err, sizeof(float *) * (size_t)P * S) == cudaSuccess;
     ok = ok && cudaMemcpy(sg->tiles, tiles.data(), sizeof(SegTile) * tiles.size(), cudaMemcpyHostToDevice) == cudaSuccess;
+    if (S <= kSegScanMax) {
+        starts.push_back(SegStart{(uint64_t)tiles.size(), 0, 0u, {0u, 0u, 0u}}); // end marker
+        ok = ok && cudaMalloc(&sg->starts, sizeof(SegStart) * starts.size()) == cudaSuccess;
+        ok = ok && cudaMemcpy(sg->starts, starts.data(), sizeof(SegStart) * starts.size(), cudaMemcpyHostToDevice) == cudaSuccess;
+    }
     ok = ok && cudaMemcpy(sg->numel, numel, sizeof(uint64_t) * S, cudaMemcpyHostToDevice) == cudaSuccess;
     ok = ok && cudaMemcpy(sg->grad, grad, sizeof(float *) * (size_t)P * S, cudaMemcpyHostToDevice) == cudaSuccess;
     ok = ok && cudaMemcpy(sg->w, w, sizeof(float *) * w_count, cudaMemcpyHostToDevice) == cudaSuccess;
@@ -1025,6 +1023,7 @@ extern "C" int a2sgd_segments_destroy(a2sgd_segments *sg)
     if (!sg) return A2SGD_OK;
     DeviceGuard guard(sg->ctx->device);
     cudaFree(sg->tiles);
+    cudaFree(sg->starts);
     cudaFree(sg->numel);
     cudaFree(sg->grad);
     cudaFree(sg->err);
@@ -1034,7 +1033,64 @@ extern "C" int a2sgd_segments_destroy(a2sgd_segments *sg)
     return A2SGD_OK;
 }
 
-static int step_segments_impl(a2sgd_ctx *c, a2sgd_segments *sg, float lr, const float *lr_per_segment, void *stream);
+static SegTables seg_tables(const a2sgd_segments *sg, const float *lr_per_segment)
+{
+    SegTables t{};
+    t.tiles = sg->tiles;
+    t.starts = sg->starts;
+    t.n_tiles = sg->n_tiles;
+    t.numel = sg->numel;
+    t.grad = sg->grad;
+    t.err = sg->err;
+    t.w = sg->w;
+    t.S = sg->S;
+    t.w_replicated = sg->replicated ? 1u : 0u;
+    t.lr_per_segment = lr_per_segment;
+    return t;
+}
+
+static int launch_encode_segments(a2sgd_ctx *c, a2sgd_segments *sg, float *local_means,
+                                  unsigned long long *pos_counts, float *global_means, cudaStream_t s)
+{
+    SegTables t = seg_tables(sg, nullptr);
+    EncodeArgs a = make_encode_args(c, nullptr, 0, nullptr, 0, local_means, pos_counts, nullptr, global_means);
+    const void *fn = !c->alg1 ? (const void *)k_encode_segments<true> : (const void *)k_encode_segments<false>;
+    const uint64_t slots = (uint64_t)c->sm_count * occupancy(c, fn) * kWavesK1;
+    uint64_t G = std::max<uint64_t>(1, slots / c->P);
+    G = std::min<uint64_t>(std::min<uint64_t>(G, sg->n_tiles), c->g_alloc);
+    void *params[] = {&a, &t};
+    A2_CUDA(launch_pdl(fn, dim3((unsigned)G, c->P), params, s));
+    return A2SGD_OK;
+}
+
+static int launch_decode_segments(a2sgd_ctx *c, a2sgd_segments *sg, const float *local_means,
+                                  const float *global_means, float lr, const float *lr_per_segment, cudaStream_t s)
+{
+    const bool ef = !c->alg1;
+    const bool store = ef || sg->has_err;
+    SegTables t = seg_tables(sg, lr_per_segment);
+    DecodeArgs a = make_decode_args(c, nullptr, sg->replicated ? 1 : 0, nullptr, 0, nullptr, 0, local_means,
+                                    global_means, lr);
+    const void *fn = ef ? select_decode_segments_p<true, true>(c->P)
+                        : store ? select_decode_segments_p<false, true>(c->P)
+                                : select_decode_segments_p<false, false>(c->P);
+    const uint64_t grid = std::min<uint64_t>(sg->n_tiles, 0x7fffffffu);
+    void *params[] = {&a, &t};
+    A2_CUDA(launch_pdl(fn, dim3((unsigned)grid), params, s));
+    return A2SGD_OK;
+}
+
+static int step_segments_impl(a2sgd_ctx *c, a2sgd_segments *sg, float lr, const float *lr_per_segment, void *stream)
+{
+    if (!c || !sg || sg->ctx != c) return A2SGD_ERR_ARG;
+    if (lr_per_segment && !device_pointer_ok(c, lr_per_segment)) return A2SGD_ERR_ARG;
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return A2SGD_ERR_CUDA;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const int rc = launch_encode_segments(c, sg, c->local_means, c->pos_counts, c->global_means, s);
+    if (rc) return rc;
+    return launch_decode_segments(c, sg, c->local_means, c->global_means, lr, lr_per_segment, s);
+}
 
 extern "C" int a2sgd_step_segments(a2sgd_ctx *c, a2sgd_segments *sg, float lr, void *stream)
 {
@@ -1047,45 +1103,34 @@ extern "C" int a2sgd_step_segments_lr(a2sgd_ctx *c, a2sgd_segments *sg, const fl
     return step_segments_impl(c, sg, 0.0f, lr_per_segment, stream);
 }
 
-static int step_segments_impl(a2sgd_ctx *c, a2sgd_segments *sg, float lr, const float *lr_per_segment, void *stream)
+extern "C" int a2sgd_encode_segments(a2sgd_ctx *c, a2sgd_segments *sg, float *local_means, uint64_t *pos_counts,
+                                     void *stream)
 {
-    if (!c || !sg || sg->ctx != c) return A2SGD_ERR_ARG;
+    if (!c || !sg || sg->ctx != c || !local_means) return A2SGD_ERR_ARG;
+    if (!aligned(local_means, 4) || (pos_counts && !aligned(pos_counts, 8))) return A2SGD_ERR_ALIGN;
+    if (!device_pointer_ok(c, local_means) || !device_pointer_ok(c, pos_counts)) return A2SGD_ERR_ARG;
     DeviceGuard guard(c->device);
     if (!guard.ok) return A2SGD_ERR_CUDA;
-    cudaStream_t s = static_cast<cudaStream_t>(stream);
-    const bool ef = !c->alg1;
-    const bool store = ef || sg->has_err;
-    SegTables t{};
-    t.tiles = sg->tiles;
-    t.n_tiles = sg->n_tiles;
-    t.numel = sg->numel;
-    t.grad = sg->grad;
-    t.err = sg->err;
-    t.w = sg->w;
-    t.S = sg->S;
-    t.w_replicated = sg->replicated ? 1u : 0u;
-    t.lr_per_segment = lr_per_segment;
-    {
-        EncodeArgs a = make_encode_args(c, nullptr, 0, nullptr, 0, c->local_means, c->pos_counts, nullptr,
-                                        c->global_means);
-        const void *fn = ef ? (const void *)k_encode_segments<true> : (const void *)k_encode_segments<false>;
-        const uint64_t slots = (uint64_t)c->sm_count * occupancy(c, fn) * A2SGD_WAVES_K1;
-        uint64_t G = std::max<uint64_t>(1, slots / c->P);
-        G = std::min<uint64_t>(std::min<uint64_t>(G, sg->n_tiles), c->g_alloc);
-        void *params[] = {&a, &t};
-        A2_CUDA(launch_pdl(fn, dim3((unsigned)G, c->P), params, s));
-    }
-    {
-        DecodeArgs a = make_decode_args(c, nullptr, sg->replicated ? 1 : 0, nullptr, 0, nullptr, 0, c->local_means,
-                                        c->global_means, lr);
-        const void *fn = ef ? select_decode_segments_p<true, true>(c->P)
-                            : store ? select_decode_segments_p<false, true>(c->P)
-                                    : select_decode_segments_p<false, false>(c->P);
-        const uint64_t grid = std::min<uint64_t>(sg->n_tiles, 0x7fffffffu);
-        void *params[] = {&a, &t};
-        A2_CUDA(launch_pdl(fn, dim3((unsigned)grid), params, s));
-    }
-    return A2SGD_OK;
+    return launch_encode_segments(c, sg, local_means, reinterpret_cast<unsigned long long *>(pos_counts), nullptr,
+                                  static_cast<cudaStream_t>(stream));
+}
+
+extern "C" int a2sgd_decode_update_segments(a2sgd_ctx *c, a2sgd_segments *sg, const float *local_means,
+                                            const float *global_means, float lr, const float *lr_per_segment,
+                                            void *stream)
+{
+    if (!c || !sg || sg->ctx != c || !global_means) return A2SGD_ERR_ARG;
+    if (c->alg1 && !local_means) return A2SGD_ERR_ARG;
+    if (!aligned(global_means, 4) || (local_means && !aligned(local_means, 4)) ||
+        (lr_per_segment && !aligned(lr_per_segment, 4)))
+        return A2SGD_ERR_ALIGN;
+    if (!device_pointer_ok(c, global_means) || !device_pointer_ok(c, local_means) ||
+        !device_pointer_ok(c, lr_per_segment))
+        return A2SGD_ERR_ARG;
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return A2SGD_ERR_CUDA;
+    return launch_decode_segments(c, sg, local_means, global_means, lr, lr_per_segment,
+                                  static_cast<cudaStream_t>(stream));
 }
 
 extern "C" int a2sgd_step_host(a2sgd_ctx *c, float *w, int64_t w_stride, const float *grad_host,
@@ -1148,12 +1193,12 @@ extern "C" int a2sgd_launch_info(a2sgd_ctx *c, int64_t w_stride, uint32_t out[5]
     // geometry for best-aligned buffers (what a caller that pads rows to 128 bytes gets)
     const bool ef = !c->alg1;
     const bool shared = w_stride == 0 || c->P == 1;
-    const int vw = A2SGD_MAX_VW >= 8 ? 8 : 4;
+    const int vw = kMaxVecWidth >= 8 ? 8 : 4;
     const uint64_t items = (c->n + vw - 1) / vw;
-    out[0] = std::min(per_worker_grid(c, occupancy(c, select_encode(ef, false, vw)), items, A2SGD_WAVES_K1),
+    out[0] = std::min(per_worker_grid(c, occupancy(c, select_encode(ef, false, vw)), items, kWavesK1),
                       c->g_alloc) * c->P;
-    out[1] = shared ? flat_grid(c, occupancy(c, select_decode_shared(ef, true, c->P, vw)), items, A2SGD_WAVES_K3)
-                    : per_worker_grid(c, occupancy(c, select_decode_repl(ef, true, vw)), items, A2SGD_WAVES_K3) * c->P;
+    out[1] = shared ? flat_grid(c, occupancy(c, select_decode_shared(ef, true, c->P, vw)), items, kWavesK3)
+                    : per_worker_grid(c, occupancy(c, select_decode_repl(ef, true, vw)), items, kWavesK3) * c->P;
     out[2] = kBlock;
     out[3] = 0;
     if (!(c->flags & A2SGD_FORCE_TWO_PASS)) {

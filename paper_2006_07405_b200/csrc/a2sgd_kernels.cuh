@@ -17,8 +17,8 @@
 // lets the hardware CTA scheduler even out SMs that stream at different
 // speeds (the host picks the grid; the loops here accept any grid).
 //
-// Summation.  Within one unrolled batch a thread adds non-negative fp32
-// values pairwise (depth <= 4, relative error <= 4 * 2^-24 of the batch sum);
+// Summation.  Within one unrolled batch (8 elements) a thread adds non-negative
+// fp32 values pairwise (depth 3, relative error <= 3 * 2^-24 of the batch sum);
 // everything above that level — the thread's running sum, the warp and block
 // trees, the cross-CTA combine — is fp64 in a fixed order.  Counts are
 // integers.  No floating-point atomics: each CTA stores one partial, and the
@@ -392,7 +392,9 @@ __global__ void __launch_bounds__(kBlock) k_encode_vec(EncodeArgs a)
     pdl_release_next_grid();
 
     constexpr int LPW = 32 / VW;  // lanes per mask word
-    constexpr int U = 16 / VW;    // vectors per trip: 16 elements per thread per batch
+    constexpr int U = 8 / VW;     // vectors per trip: 8 elements per thread per batch.  One 256-bit vector of g
+                                  // and of e per trip keeps the kernel at 48 registers (5 CTAs per SM); two per
+                                  // trip (64 B + 64 B in flight per thread, 4 CTAs per SM) measured 1-2 % slower
     __shared__ double sh_d[2][kWarps];
     __shared__ unsigned long long sh_n[kWarps];
     __shared__ int sh_flag;

@@ -26,8 +26,21 @@ struct __align__(16) SegTile {
     uint64_t offset; // first element of the tile inside the tensor
 };
 
+// First tile and access flags of a tensor; one entry per tensor plus an end marker.  The decode
+// kernel finds its tensor by scanning this small table (L1-resident: every CTA reads the same
+// entries) instead of reading a per-tile descriptor, which would be a fresh L2 access in front of
+// every CTA's data loads.
+struct __align__(16) SegStart {
+    uint64_t first_tile;
+    uint64_t numel;
+    uint32_t flags;
+    uint32_t pad[3];
+};
+constexpr uint32_t kSegScanMax = 4096; // tensors up to which the decode kernel scans SegStart (else: tile table)
+
 struct SegTables {
     const SegTile *tiles;
+    const SegStart *starts; // [S + 1] or nullptr (S > kSegScanMax)
     uint64_t n_tiles;
     const uint64_t *numel;      // [S]
     const float *const *grad;   // [P][S] device pointers, worker-major
@@ -37,6 +50,14 @@ struct SegTables {
     uint32_t w_replicated;
     const float *lr_per_segment; // [S] device, or nullptr: one learning rate for the whole model
 };
+
+// An entry of a pointer table through the read-only (L1-cached) path: the tables are small and every
+// CTA of a tensor reads the same entries, while the data streams bypass L1.
+template <typename T>
+__device__ __forceinline__ T *ld_ptr(T *const *slot)
+{
+    return reinterpret_cast<T *>(__ldg(reinterpret_cast<const unsigned long long *>(slot)));
+}
 
 // K1 over a segment list.  grid = (G, P); CTA x walks tiles x, x + G, ...
 template <bool EF>
@@ -115,33 +136,67 @@ __global__ void __launch_bounds__(kBlock) k_decode_segments(DecodeArgs a, SegTab
         for (uint32_t p = threadIdx.x; p < P; p += kBlock) sh_c[p] = worker_const<EF>(a, p, m_pos, m_neg);
         __syncthreads();
     }
+    __shared__ SegTile sh_tile;
+    __shared__ uint64_t sh_numel;
     for (uint64_t tile = blockIdx.x; tile < t.n_tiles; tile += gridDim.x) {
-        const SegTile d = t.tiles[tile];
-        const uint64_t n_s = t.numel[d.seg];
+        SegTile d;
+        uint64_t n_s;
+        if (t.starts) {
+            for (uint32_t sg = threadIdx.x; sg < t.S; sg += kBlock) {
+                const uint64_t lo = __ldg(&t.starts[sg].first_tile), hi = __ldg(&t.starts[sg + 1].first_tile);
+                if (tile >= lo && tile < hi) {
+                    sh_tile = SegTile{sg, __ldg(&t.starts[sg].flags), (tile - lo) * kSegTile};
+                    sh_numel = __ldg(&t.starts[sg].numel);
+                }
+            }
+            __syncthreads();
+            d = sh_tile;
+            n_s = sh_numel;
+            if (tile + gridDim.x < t.n_tiles) __syncthreads(); // the slots are rewritten in the next trip
+        } else {
+            d = t.tiles[tile];
+            n_s = __ldg(t.numel + d.seg);
+        }
         const uint64_t i = d.offset + (uint64_t)threadIdx.x * kSegVW;
         // layer-wise learning rates (e.g. LARS, which the paper uses for VGG-16): one per tensor
         const float lr = t.lr_per_segment ? __ldg(t.lr_per_segment + d.seg) : a.lr;
         const float scale = repl ? -lr : -lr / (float)P;
         if ((d.flags & kSegFlagVec) && i + kSegVW <= n_s) {
             if (PT > 0 && !repl) {
+                // workers in batches of four, as in the flat kernel: all loads of a batch are issued
+                // before its first store, and the register count stays low enough for two CTAs per SM
                 constexpr int PP = PT > 0 ? PT : 1;
-                Vec<kSegVW> gv[PP], ev[PP];
-                float *wp = t.w[d.seg] + i;
-                const Vec<kSegVW> wv = ld_vec<kSegVW>(wp);
+                constexpr int PB = PP < 4 ? PP : 4;
+                // every pointer of the tile is fetched before the first data access: a pointer load
+                // placed after a store could not be moved above it
+                const float *gp[PP];
+                float *ep[PP];
+                float *wp = ld_ptr(t.w + d.seg) + i;
 #pragma unroll
-                for (int p = 0; p < PP; ++p) gv[p] = ld_vec<kSegVW>(t.grad[(uint64_t)p * t.S + d.seg] + i);
-                if (EF) {
+                for (int p = 0; p < PP; ++p) gp[p] = ld_ptr(t.grad + (uint64_t)p * t.S + d.seg) + i;
+                if (EF || STORE) {
 #pragma unroll
-                    for (int p = 0; p < PP; ++p) ev[p] = ld_vec<kSegVW>(t.err[(uint64_t)p * t.S + d.seg] + i);
+                    for (int p = 0; p < PP; ++p) ep[p] = ld_ptr(t.err + (uint64_t)p * t.S + d.seg) + i;
                 }
+                const Vec<kSegVW> wv = ld_vec<kSegVW>(wp);
                 Vec<kSegVW> sum = zero_vec<kSegVW>();
 #pragma unroll
-                for (int p = 0; p < PP; ++p) {
-                    const Vec<kSegVW> v = EF ? add_vec<kSegVW>(gv[p], ev[p]) : gv[p];
-                    Vec<kSegVW> gh, rs;
-                    decode_vec<EF, kSegVW>(v, worker_const<EF>(a, p, m_pos, m_neg), gh, rs);
-                    sum = add_vec<kSegVW>(sum, gh);
-                    if (STORE) st_vec<kSegVW>(t.err[(uint64_t)p * t.S + d.seg] + i, rs);
+                for (int p0 = 0; p0 < PP; p0 += PB) {
+                    Vec<kSegVW> gv[PB], ev[PB];
+#pragma unroll
+                    for (int q = 0; q < PB; ++q) gv[q] = ld_vec<kSegVW>(gp[p0 + q]);
+                    if (EF) {
+#pragma unroll
+                        for (int q = 0; q < PB; ++q) ev[q] = ld_vec<kSegVW>(ep[p0 + q]);
+                    }
+#pragma unroll
+                    for (int q = 0; q < PB; ++q) {
+                        const Vec<kSegVW> v = EF ? add_vec<kSegVW>(gv[q], ev[q]) : gv[q];
+                        Vec<kSegVW> gh, rs;
+                        decode_vec<EF, kSegVW>(v, worker_const<EF>(a, p0 + q, m_pos, m_neg), gh, rs);
+                        sum = add_vec<kSegVW>(sum, gh);
+                        if (STORE) st_vec<kSegVW>(ep[p0 + q], rs);
+                    }
                 }
                 st_vec<kSegVW>(wp, axpy_vec<kSegVW>(scale, sum, wv));
             } else {
