@@ -68,11 +68,16 @@ enum a2sgd_status {
     A2SGD_ERR_ARG = -1,       /* NULL pointer, n or P out of range, stride < n, bad flag */
     A2SGD_ERR_ALIGN = -2,     /* a float pointer that is not 4-byte aligned */
     A2SGD_ERR_CUDA = -3,      /* a CUDA runtime call failed */
-    A2SGD_ERR_TIMEOUT = -4,   /* a bounded device-side wait ran out (latched in the status word) */
+    A2SGD_ERR_TIMEOUT = -4,   /* a bounded device-side wait ran out (latched in the status word).  A CTA that
+                                 gives up writes nothing, and the barrier is left shut once one has, but a CTA
+                                 may still give up after the others went on: after this status w and err of
+                                 that step are undefined — restore them from a copy */
     A2SGD_ERR_NONFINITE = -5, /* a group sum was NaN or Inf (latched in the status word) */
     A2SGD_ERR_NOMEM = -6,     /* scratch allocation failed */
-    A2SGD_ERR_TOO_LARGE = -7  /* n*P exceeds what the single-launch path can hold on chip (A2SGD_FORCE_COOPERATIVE),
+    A2SGD_ERR_TOO_LARGE = -7, /* n*P exceeds what the single-launch path can hold on chip (A2SGD_FORCE_COOPERATIVE),
                                  or P > A2SGD_NOALLOC_MAX_P in a2sgd_encode_noalloc (its fixed scratch) */
+    A2SGD_ERR_BOUNDS = -8     /* A2SGD_DEBUG_CHECKS: a kernel computed an access outside the live elements of
+                                 the buffers it was given; the access was skipped (latched in the status word) */
 };
 
 enum a2sgd_flags {
@@ -96,11 +101,27 @@ enum a2sgd_flags {
                                          mask of P*n/8 bytes.  Which kernel a step launches depends on
                                          host-side state (does the buffer hold v yet?), so a captured step
                                          must not be replayed across the first step or a materialise call. */
-    A2SGD_CHECK_POINTERS = 1 << 8,    /* every call first asks the runtime whether each buffer is device (or
-                                         managed) memory usable from the context's device and returns
-                                         A2SGD_ERR_ARG otherwise, before anything is launched: a host pointer
-                                         handed to a kernel would fault the GPU.  Costs about a microsecond
-                                         per pointer per call; off by default. */
+    A2SGD_CHECK_POINTERS = 1 << 8,    /* every call that takes device buffers first asks the runtime whether each
+                                         one is device (or managed) memory usable from the context's device and
+                                         returns A2SGD_ERR_ARG otherwise, before anything is launched: a host
+                                         pointer handed to a kernel would fault the GPU.  A segment plan checks
+                                         every tensor pointer once, in a2sgd_segments_create.  Costs about a
+                                         microsecond per pointer per call; off by default. */
+    A2SGD_DEBUG_CHECKS = 1 << 10,     /* the stand-in for a memory checker where none can be run: while a call
+                                         of this context is in flight, every access its kernels make to grad, err,
+                                         w, the momentum buffer and the packed mask is first checked, on the
+                                         device, against the extents the call was given (inside the n live
+                                         elements of one row); an access that is not is skipped — loads return 0 —
+                                         and A2SGD_ERR_BOUNDS is latched for a2sgd_read_stats.  Nothing traps or
+                                         faults.  For segment lists the check is on tile and tensor indices
+                                         instead of addresses.  The extents live in one descriptor per device, so
+                                         calls of a checking context must not overlap other calls of the library
+                                         on the same device (different streams or threads).  Several times
+                                         slower; off by default. */
+    A2SGD_TEST_SHRINK_EXTENTS = 1 << 11, /* test hook for A2SGD_DEBUG_CHECKS: the extents recorded for a call are
+                                            one element per row short, so the checked kernels skip every access
+                                            that touches a row's last element and latch A2SGD_ERR_BOUNDS — the
+                                            check is seen to fire without any access ever leaving a buffer */
     A2SGD_TEST_BARRIER_NEVER_OPENS = 1 << 9 /* test hook: the single-launch path waits for one arrival more
                                                than its grid has, with a ~0.2 ms limit, so every CTA gives up,
                                                writes nothing and A2SGD_ERR_TIMEOUT is latched */
@@ -188,9 +209,9 @@ int a2sgd_step_momentum(a2sgd_ctx *ctx, float *w, int64_t w_stride, float *mom, 
                         const float *grad, int64_t grad_stride, float *err, int64_t err_stride,
                         float lr, float beta, float weight_decay, void *stream);
 
-/* a2sgd_step with the fresh gradients stored as bfloat16 (the paper remarks that the method
- * "can be further integrated with quantization"; a bfloat16 gradient is the common case of a
- * mixed-precision backward pass).  grad: [P] vectors of n bfloat16 values (raw uint16 bit
+/* a2sgd_step with the fresh gradients stored as bfloat16 (Section 1 of the paper names the
+ * combination with quantisation as a natural extension; a bfloat16 gradient is the common case
+ * of a mixed-precision backward pass).  grad: [P] vectors of n bfloat16 values (raw uint16 bit
  * patterns), worker stride grad_stride in ELEMENTS.  Widening bfloat16 to fp32 is exact, so the
  * result equals a2sgd_step on the widened gradients; err and w stay fp32.  Traffic drops from
  * (20P + 8) to (16P + 8) bytes per model element.  Always two launches.  The fast path needs
@@ -231,8 +252,8 @@ int a2sgd_dense_sync_reduced(a2sgd_ctx *ctx, float *w, const float *grad_sum, ui
 
 /* Segment lists: the model as S separate tensors (the way a training framework holds its
  * parameters and gradients) instead of one flat vector.  The S tensors are treated as the
- * concatenation they would form: ONE pair of means per worker over the whole model ("for each
- * model, it traverses all gradients to compute two separate averages", Section 4.3), the same
+ * concatenation they would form: ONE pair of means per worker over the whole model (Section 4.3:
+ * the two averages are taken over all gradients of the model), the same
  * results as a2sgd_step on the flattened copy, without making that copy.
  *
  * a2sgd_segments_create records the layout once (device tables owned by the plan):

@@ -18,7 +18,7 @@ from typing import Optional, Tuple
 import torch
 
 OK = 0
-ERR_ARG, ERR_ALIGN, ERR_CUDA, ERR_TIMEOUT, ERR_NONFINITE, ERR_NOMEM, ERR_TOO_LARGE = -1, -2, -3, -4, -5, -6, -7
+ERR_ARG, ERR_ALIGN, ERR_CUDA, ERR_TIMEOUT, ERR_NONFINITE, ERR_NOMEM, ERR_TOO_LARGE, ERR_BOUNDS = -1, -2, -3, -4, -5, -6, -7, -8
 MODE_EF = 0
 MODE_ALG1 = 1
 FORCE_TWO_PASS = 1 << 4
@@ -26,6 +26,8 @@ FORCE_COOPERATIVE = 1 << 5
 DEFERRED_RESIDUAL = 1 << 7
 CHECK_POINTERS = 1 << 8
 TEST_BARRIER_NEVER_OPENS = 1 << 9
+DEBUG_CHECKS = 1 << 10
+TEST_SHRINK_EXTENTS = 1 << 11
 ROW_ALIGN_ELEMS = 32   # 128 bytes: rows that start on a cache-line boundary take the widest vector kernels
 
 _HERE = os.path.dirname(os.path.abspath(__file__))

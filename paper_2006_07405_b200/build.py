@@ -12,14 +12,17 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "liba2sgd.so")
-SOURCES = [os.path.join(CSRC, "a2sgd.cu"), os.path.join(CSRC, "a2sgd_noalloc.cu")]
-DEPENDS = SOURCES + [os.path.join(CSRC, "a2sgd_kernels.cuh"), os.path.join(ROOT, "include", "a2sgd.h")]
+SOURCES = [os.path.join(CSRC, f) for f in ("a2sgd.cu", "a2sgd_checked.cu", "a2sgd_noalloc.cu")]
+DEPENDS = SOURCES + [os.path.join(CSRC, f) for f in ("a2sgd_kernels.cuh", "a2sgd_segments.cuh", "a2sgd_select.cuh",
+                                                     "a2sgd_kernel_table.h", "a2sgd_debug_check.h")] \
+    + [os.path.join(ROOT, "include", "a2sgd.h")]
 
-NVCC_FLAGS = [
+COMPILE_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
     "--ftz=false", "--prec-div=true", "--prec-sqrt=true",   # a flushed subnormal would change its sign group
-    "-shared", "-Xcompiler", "-fPIC", "-cudart", "static",
+    "-Xcompiler", "-fPIC",
 ]
+LINK_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-shared", "-Xcompiler", "-fPIC", "-cudart", "static"]
 
 
 def nvcc() -> str:
@@ -38,10 +41,26 @@ def is_stale() -> bool:
 
 def build(force: bool = False, verbose: bool = False) -> str:
     if force or is_stale():
+        # the translation units are compiled side by side (the production and the checked copy of
+        # the kernels take about the same time), then linked; the library is replaced atomically
+        from concurrent.futures import ThreadPoolExecutor
+        objs = [f"{LIB}.{os.getpid()}.{i}.o" for i in range(len(SOURCES))]
+
+        def compile_one(job):
+            src, obj = job
+            cmd = [nvcc()] + COMPILE_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-c", "-o", obj, src]
+            subprocess.check_call(cmd)
+
         tmp = f"{LIB}.{os.getpid()}.tmp"
-        cmd = [nvcc()] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-o", tmp] + SOURCES
-        subprocess.check_call(cmd)
-        os.replace(tmp, LIB)
+        try:
+            with ThreadPoolExecutor(max_workers=len(SOURCES)) as pool:
+                list(pool.map(compile_one, zip(SOURCES, objs)))
+            subprocess.check_call([nvcc()] + LINK_FLAGS + ["-o", tmp] + objs)
+            os.replace(tmp, LIB)
+        finally:
+            for f in objs + [tmp]:
+                if os.path.exists(f):
+                    os.remove(f)
     return LIB
 
 

@@ -10,10 +10,18 @@
 #include <unordered_map>
 #include <vector>
 
+#include "a2sgd_kernel_table.h"
+#define A2SGD_NS a2sgd
+#define A2SGD_CHECKED 0
 #include "a2sgd_kernels.cuh"
 #include "a2sgd_segments.cuh"
+#include "a2sgd_select.cuh"
 
 using namespace a2sgd;
+
+// The checked copy of the kernels lives in its own translation unit (a2sgd_checked.cu).
+const a2sgd_kernel_table *a2sgd_checked_kernels();
+cudaError_t a2sgd_checked_arm(const void *descriptor, size_t bytes, cudaStream_t stream);
 
 // Grid shapes (measured on B200, CUDA events, c2-c5 workloads):
 //  * decode: one vector per thread, as many CTAs as that takes.  A persistent grid of
@@ -53,6 +61,7 @@ struct a2sgd_ctx {
     uint32_t *sign_mask = nullptr; // [P][ceil(n/32)]
     float *prev_means = nullptr;   // [2]
     bool err_holds_v = false;      // the caller's error buffer currently holds v, not e
+    const a2sgd_kernel_table *k = nullptr; // production kernels, or the checked copy (A2SGD_DEBUG_CHECKS)
     // resident CTAs per SM of every kernel instance used so far (occupancy API, cached)
     std::unordered_map<const void *, int> occ;
 };
@@ -161,170 +170,12 @@ inline uint32_t flat_grid(const a2sgd_ctx *c, int occ, uint64_t items, int waves
     return (uint32_t)std::min<uint64_t>(std::min(slots, need), 0x7fffffffu);
 }
 
-// ---------------------------------------------------------------- kernel selection
-const void *select_encode(bool ef, bool mask, int vw)
-{
-#define A2_PICK(EF, MASK)                                                               \
-    (vw == 8 ? (const void *)k_encode_vec<EF, MASK, 8>                                  \
-             : vw == 4 ? (const void *)k_encode_vec<EF, MASK, 4> : (const void *)k_encode_scalar<EF, MASK>)
-    if (ef) return mask ? A2_PICK(true, true) : A2_PICK(true, false);
-    return mask ? A2_PICK(false, true) : A2_PICK(false, false);
-#undef A2_PICK
-}
-
-template <bool EF, bool STORE, int VW, bool MOM>
-const void *select_decode_shared_p(uint32_t P)
-{
-    switch (P) {
-    case 1: return (const void *)k_decode_shared_vec<EF, STORE, 1, VW, 0, MOM>;
-    case 2: return (const void *)k_decode_shared_vec<EF, STORE, 2, VW, 0, MOM>;
-    case 4: return (const void *)k_decode_shared_vec<EF, STORE, 4, VW, 0, MOM>;
-    case 8: return (const void *)k_decode_shared_vec<EF, STORE, 8, VW, 0, MOM>;
-    default: return (const void *)k_decode_shared_vec<EF, STORE, 0, VW, 0, MOM>;
-    }
-}
-
-template <bool MOM>
-const void *select_decode_shared_m(bool ef, bool store, uint32_t P, int vw)
-{
-    if (vw == 8) {
-        if (ef) return select_decode_shared_p<true, true, 8, MOM>(P);
-        return store ? select_decode_shared_p<false, true, 8, MOM>(P) : select_decode_shared_p<false, false, 8, MOM>(P);
-    }
-    if (ef) return select_decode_shared_p<true, true, 4, MOM>(P);
-    return store ? select_decode_shared_p<false, true, 4, MOM>(P) : select_decode_shared_p<false, false, 4, MOM>(P);
-}
-
-const void *select_decode_shared(bool ef, bool store, uint32_t P, int vw, bool mom = false)
-{
-    return mom ? select_decode_shared_m<true>(ef, store, P, vw) : select_decode_shared_m<false>(ef, store, P, vw);
-}
-
-template <bool MOM>
-const void *select_decode_repl_m(bool ef, bool store, int vw)
-{
-    if (vw == 8) {
-        if (ef) return (const void *)k_decode_repl_vec<true, true, 8, 0, MOM>;
-        return store ? (const void *)k_decode_repl_vec<false, true, 8, 0, MOM>
-                     : (const void *)k_decode_repl_vec<false, false, 8, 0, MOM>;
-    }
-    if (ef) return (const void *)k_decode_repl_vec<true, true, 4, 0, MOM>;
-    return store ? (const void *)k_decode_repl_vec<false, true, 4, 0, MOM>
-                 : (const void *)k_decode_repl_vec<false, false, 4, 0, MOM>;
-}
-
-const void *select_decode_repl(bool ef, bool store, int vw, bool mom = false)
-{
-    return mom ? select_decode_repl_m<true>(ef, store, vw) : select_decode_repl_m<false>(ef, store, vw);
-}
-
-const void *select_decode_scalar(bool ef, bool store, bool mom = false)
-{
-    if (mom) {
-        if (ef) return (const void *)k_decode_scalar<true, true, 0, true>;
-        return store ? (const void *)k_decode_scalar<false, true, 0, true> : (const void *)k_decode_scalar<false, false, 0, true>;
-    }
-    if (ef) return (const void *)k_decode_scalar<true, true>;
-    return store ? (const void *)k_decode_scalar<false, true> : (const void *)k_decode_scalar<false, false>;
-}
-
-// 16-bit gradient rows (GT = 1 bfloat16, 2 half): 8-element (128-bit) vectors or scalar accesses
-template <bool EF, bool STORE, int GT>
-const void *select_decode_shared_lowp_p(uint32_t P)
-{
-    switch (P) {
-    case 1: return (const void *)k_decode_shared_vec<EF, STORE, 1, 8, GT>;
-    case 2: return (const void *)k_decode_shared_vec<EF, STORE, 2, 8, GT>;
-    case 4: return (const void *)k_decode_shared_vec<EF, STORE, 4, 8, GT>;
-    case 8: return (const void *)k_decode_shared_vec<EF, STORE, 8, 8, GT>;
-    default: return (const void *)k_decode_shared_vec<EF, STORE, 0, 8, GT>;
-    }
-}
-
-template <int GT>
-const void *select_encode_lowp(bool ef, int vw)
-{
-    if (vw == 8) return ef ? (const void *)k_encode_vec<true, false, 8, GT> : (const void *)k_encode_vec<false, false, 8, GT>;
-    return ef ? (const void *)k_encode_scalar<true, false, GT> : (const void *)k_encode_scalar<false, false, GT>;
-}
-
-template <int GT>
-const void *select_decode_lowp(bool ef, bool store, bool shared, uint32_t P, int vw)
-{
-    if (vw == 8 && shared) {
-        if (ef) return select_decode_shared_lowp_p<true, true, GT>(P);
-        return store ? select_decode_shared_lowp_p<false, true, GT>(P) : select_decode_shared_lowp_p<false, false, GT>(P);
-    }
-    if (vw == 8) {
-        if (ef) return (const void *)k_decode_repl_vec<true, true, 8, GT>;
-        return store ? (const void *)k_decode_repl_vec<false, true, 8, GT> : (const void *)k_decode_repl_vec<false, false, 8, GT>;
-    }
-    if (ef) return (const void *)k_decode_scalar<true, true, GT>;
-    return store ? (const void *)k_decode_scalar<false, true, GT> : (const void *)k_decode_scalar<false, false, GT>;
-}
-
 // a 16-bit row allows 8-element vectors when it is 16-byte aligned with a stride multiple of 8
 inline int vec_width_bf16(const void *p, int64_t stride, uint32_t P)
 {
     return (aligned(p, 16) && (P == 1 || stride % 8 == 0)) ? 8 : 0;
 }
 
-template <int VW, bool REPL>
-const void *select_dense_p(uint32_t P)
-{
-    switch (P) {
-    case 1: return (const void *)k_dense_sync_vec<1, VW, REPL>;
-    case 2: return (const void *)k_dense_sync_vec<2, VW, REPL>;
-    case 4: return (const void *)k_dense_sync_vec<4, VW, REPL>;
-    case 8: return (const void *)k_dense_sync_vec<8, VW, REPL>;
-    default: return (const void *)k_dense_sync_vec<0, VW, REPL>;
-    }
-}
-
-const void *select_dense(uint32_t P, int vw, bool repl)
-{
-    if (vw == 8) return repl ? select_dense_p<8, true>(P) : select_dense_p<8, false>(P);
-    if (vw == 4) return repl ? select_dense_p<4, true>(P) : select_dense_p<4, false>(P);
-    return (const void *)k_dense_sync_scalar;
-}
-
-template <bool EF, bool STORE, bool SHARED>
-const void *select_coop_p(uint32_t P)
-{
-    switch (P) {
-    case 1: return (const void *)k_step_coop<EF, STORE, 1, SHARED>;
-    case 2: return (const void *)k_step_coop<EF, STORE, 2, SHARED>;
-    case 4: return (const void *)k_step_coop<EF, STORE, 4, SHARED>;
-    case 8: return (const void *)k_step_coop<EF, STORE, 8, SHARED>;
-    default: return nullptr;
-    }
-}
-
-template <bool EF, bool STORE, bool SHARED>
-const void *select_coop_l2_p(uint32_t P)
-{
-    switch (P) {
-    case 1: return (const void *)k_step_coop_l2<EF, STORE, 1, SHARED>;
-    case 2: return (const void *)k_step_coop_l2<EF, STORE, 2, SHARED>;
-    case 4: return (const void *)k_step_coop_l2<EF, STORE, 4, SHARED>;
-    case 8: return (const void *)k_step_coop_l2<EF, STORE, 8, SHARED>;
-    default: return nullptr;
-    }
-}
-
-const void *select_coop_l2(bool ef, bool store, bool shared, uint32_t P)
-{
-    if (ef) return shared ? select_coop_l2_p<true, true, true>(P) : select_coop_l2_p<true, true, false>(P);
-    if (store) return shared ? select_coop_l2_p<false, true, true>(P) : select_coop_l2_p<false, true, false>(P);
-    return shared ? select_coop_l2_p<false, false, true>(P) : select_coop_l2_p<false, false, false>(P);
-}
-
-const void *select_coop(bool ef, bool store, bool shared, uint32_t P)
-{
-    if (ef) return shared ? select_coop_p<true, true, true>(P) : select_coop_p<true, true, false>(P);
-    if (store) return shared ? select_coop_p<false, true, true>(P) : select_coop_p<false, true, false>(P);
-    return shared ? select_coop_p<false, false, true>(P) : select_coop_p<false, false, false>(P);
-}
 
 // ---------------------------------------------------------------- launches
 EncodeArgs make_encode_args(a2sgd_ctx *c, const float *grad, int64_t gs, const float *err, int64_t es,
@@ -388,7 +239,7 @@ int launch_encode(a2sgd_ctx *c, const float *grad, int64_t gs, const float *err,
 {
     const int vw = encode_vec_width(c, grad, gs, err, es);
     EncodeArgs a = make_encode_args(c, grad, gs, err, es, local_means, pos_counts, pos_mask, global_means);
-    const void *fn = select_encode(!c->alg1, pos_mask != nullptr, vw);
+    const void *fn = c->k->encode(!c->alg1, pos_mask != nullptr, vw);
     const uint64_t items = vw ? (c->n + vw - 1) / vw : (c->n + kScalarU - 1) / kScalarU;
     const dim3 grid(std::min(per_worker_grid(c, occupancy(c, fn), items, kWavesK1), c->g_alloc), c->P);
     void *params[] = {&a};
@@ -425,13 +276,13 @@ int launch_decode(a2sgd_ctx *c, float *w, int64_t ws, const float *grad, int64_t
     const void *fn;
     dim3 grid;
     if (vw && shared) {
-        fn = select_decode_shared(ef, store, c->P, vw, mom);
+        fn = c->k->decode_shared(ef, store, c->P, vw, mom);
         grid = dim3(flat_grid(c, occupancy(c, fn), (c->n + vw - 1) / vw, kWavesK3));
     } else if (vw) {
-        fn = select_decode_repl(ef, store, vw, mom);
+        fn = c->k->decode_repl(ef, store, vw, mom);
         grid = dim3(per_worker_grid(c, occupancy(c, fn), (c->n + vw - 1) / vw, kWavesK3), c->P);
     } else {
-        fn = select_decode_scalar(ef, store, mom);
+        fn = c->k->decode_scalar(ef, store, mom);
         const uint64_t items = (c->n + kDecScalarU - 1) / kDecScalarU; // one tile of kBlock * kDecScalarU per CTA
         grid = shared ? dim3(flat_grid(c, occupancy(c, fn), items, kWavesK3), 1)
                       : dim3(per_worker_grid(c, occupancy(c, fn), items, kWavesK3), c->P);
@@ -457,7 +308,7 @@ const void *coop_plan(a2sgd_ctx *c, bool store, bool shared, int vw, uint32_t *g
     if (!c->coop_supported || vw < 4) return nullptr;
     const bool forced = (c->flags & A2SGD_FORCE_COOPERATIVE) != 0;
     if (!forced && c->P != 1) return nullptr;
-    const void *fn = select_coop(!c->alg1, store, shared, c->P);
+    const void *fn = c->k->coop(!c->alg1, store, shared, c->P);
     if (!fn) return nullptr;
     const uint64_t n4 = (c->n + 3) / 4;
     const uint64_t need = std::max<uint64_t>(1, (n4 + kBlock - 1) / kBlock);
@@ -471,7 +322,7 @@ const void *coop_plan(a2sgd_ctx *c, bool store, bool shared, int vw, uint32_t *g
         }
     }
     if (!forced) return nullptr;
-    const void *fn2 = select_coop_l2(!c->alg1, store, shared, c->P);
+    const void *fn2 = c->k->coop_l2(!c->alg1, store, shared, c->P);
     const uint64_t rows = (uint64_t)c->P * (c->alg1 ? (store ? 2 : 1) : 2) + (shared ? 1 : c->P);
     const double footprint = (double)rows * (double)c->n * 4.0;
     if (!fn2 || footprint > 0.70 * (double)c->l2_bytes) return nullptr;
@@ -495,18 +346,6 @@ int launch_coop(a2sgd_ctx *c, const void *fn, uint32_t grid, float *w, int64_t w
     return A2SGD_OK;
 }
 
-template <bool REPL>
-const void *select_decode_deferred(uint32_t P)
-{
-    switch (P) {
-    case 1: return (const void *)k_decode_deferred<1, REPL>;
-    case 2: return (const void *)k_decode_deferred<2, REPL>;
-    case 4: return (const void *)k_decode_deferred<4, REPL>;
-    case 8: return (const void *)k_decode_deferred<8, REPL>;
-    default: return (const void *)k_decode_deferred<0, REPL>;
-    }
-}
-
 // One step in the deferred-residual representation (see k_encode_vec / k_decode_deferred).
 int deferred_step(a2sgd_ctx *c, float *w, int64_t ws, const float *grad, int64_t gs, float *err, int64_t es,
                   float lr, cudaStream_t s)
@@ -518,8 +357,7 @@ int deferred_step(a2sgd_ctx *c, float *w, int64_t ws, const float *grad, int64_t
         EncodeArgs a = make_encode_args(c, grad, gs, err, es, c->local_means, c->pos_counts, c->sign_mask,
                                         c->global_means);
         a.prev_means = c->prev_means;
-        const void *fn = c->err_holds_v ? (const void *)k_encode_vec<true, true, 8, false, 2>
-                                        : (const void *)k_encode_vec<true, true, 8, false, 1>;
+        const void *fn = c->k->encode_deferred(c->err_holds_v);
         const dim3 grid(std::min(per_worker_grid(c, occupancy(c, fn), (c->n + 7) / 8, kWavesK1Deferred), c->g_alloc), c->P);
         void *params[] = {&a};
         A2_CUDA(launch_pdl(fn, grid, params, s));
@@ -536,7 +374,7 @@ int deferred_step(a2sgd_ctx *c, float *w, int64_t ws, const float *grad, int64_t
         a.global_means = c->global_means;
         a.prev_means = c->prev_means;
         a.lr = lr;
-        const void *fn = ws == 0 ? select_decode_deferred<false>(c->P) : select_decode_deferred<true>(c->P);
+        const void *fn = c->k->decode_deferred(ws != 0, c->P);
         const dim3 grid(flat_grid(c, occupancy(c, fn), std::max<uint64_t>(1, (c->n / 32) * 4), kWavesK3));
         void *params[] = {&a};
         A2_CUDA(launch_pdl(fn, grid, params, s));
@@ -558,6 +396,44 @@ bool device_pointer_ok(const a2sgd_ctx *c, const void *p)
     return attr.type == cudaMemoryTypeDevice && attr.device == c->device;
 }
 
+// A2SGD_DEBUG_CHECKS: for the duration of one call's launches the device-side descriptor of the
+// checked kernels holds the extents of the call's buffers; the destructor switches it off again
+// (stream-ordered after the kernels).  Buffers are added as `rows` rows of `n` elements of `elem`
+// bytes, `stride` elements apart.
+struct DebugScope {
+    a2sgd_ctx *c;
+    cudaStream_t s;
+    DebugChecks d{};
+    bool armed = false;
+    DebugScope(a2sgd_ctx *ctx, cudaStream_t stream) : c(ctx), s(stream) {}
+    void add(const void *base, uint64_t rows, int64_t stride, uint64_t n, uint32_t elem)
+    {
+        if (!(c->flags & A2SGD_DEBUG_CHECKS) || !base || d.count >= kDebugMaxRanges) return;
+        DebugRange &r = d.range[d.count++];
+        r.base = (uint64_t)reinterpret_cast<uintptr_t>(base);
+        r.rows = rows;
+        r.stride_bytes = rows > 1 ? (uint64_t)stride * elem : 0;
+        r.row_bytes = n * elem;
+        if ((c->flags & A2SGD_TEST_SHRINK_EXTENTS) && n > 1) r.row_bytes -= elem;
+    }
+    // mode 1: the address ranges added so far; mode 2: index checks only (segment lists)
+    bool arm(int mode)
+    {
+        if (!(c->flags & A2SGD_DEBUG_CHECKS)) return true;
+        d.on = mode;
+        d.status = c->status;
+        armed = a2sgd_checked_arm(&d, sizeof(d), s) == cudaSuccess;
+        if (!armed) (void)cudaGetLastError();
+        return armed;
+    }
+    ~DebugScope()
+    {
+        if (!armed) return;
+        const DebugChecks off{};
+        if (a2sgd_checked_arm(&off, sizeof(off), s) != cudaSuccess) (void)cudaGetLastError();
+    }
+};
+
 int check_common(const a2sgd_ctx *c, const float *grad, int64_t gs, const float *err, int64_t es,
                  bool err_required)
 {
@@ -578,7 +454,8 @@ extern "C" int a2sgd_create(a2sgd_ctx **out, uint64_t n, uint32_t P, int device,
     if (!out) return A2SGD_ERR_ARG;
     *out = nullptr;
     const uint32_t known = A2SGD_MODE_ALG1 | A2SGD_FORCE_TWO_PASS | A2SGD_FORCE_COOPERATIVE |
-                           A2SGD_TEST_BARRIER_NEVER_OPENS | A2SGD_DEFERRED_RESIDUAL | A2SGD_CHECK_POINTERS;
+                           A2SGD_TEST_BARRIER_NEVER_OPENS | A2SGD_DEFERRED_RESIDUAL | A2SGD_CHECK_POINTERS |
+                           A2SGD_DEBUG_CHECKS | A2SGD_TEST_SHRINK_EXTENTS;
     if ((flags & A2SGD_DEFERRED_RESIDUAL) && (flags & (A2SGD_MODE_ALG1 | A2SGD_FORCE_COOPERATIVE))) return A2SGD_ERR_ARG;
     if (n == 0 || n >= (1ull << 40) || P == 0 || P > (uint32_t)kMaxP || (flags & ~known)) return A2SGD_ERR_ARG;
     if ((flags & A2SGD_FORCE_TWO_PASS) && (flags & A2SGD_FORCE_COOPERATIVE)) return A2SGD_ERR_ARG;
@@ -595,6 +472,8 @@ extern "C" int a2sgd_create(a2sgd_ctx **out, uint64_t n, uint32_t P, int device,
     c->device = device;
     c->flags = flags;
     c->alg1 = (flags & A2SGD_MODE_ALG1) != 0;
+    static const a2sgd_kernel_table production = a2sgd::kernel_table();
+    c->k = (flags & A2SGD_DEBUG_CHECKS) ? a2sgd_checked_kernels() : &production;
     if (cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, device) != cudaSuccess) {
         delete c;
         return A2SGD_ERR_CUDA;
@@ -671,6 +550,11 @@ extern "C" int a2sgd_encode(a2sgd_ctx *c, const float *grad, int64_t grad_stride
         return A2SGD_ERR_ARG;
     DeviceGuard guard(c->device);
     if (!guard.ok) return A2SGD_ERR_CUDA;
+    DebugScope dbg(c, static_cast<cudaStream_t>(stream));
+    dbg.add(grad, c->P, grad_stride, c->n, 4);
+    if (!c->alg1) dbg.add(err, c->P, err_stride, c->n, 4);
+    dbg.add(pos_mask, c->P, (int64_t)((c->n + 31) / 32), (c->n + 31) / 32, 4);
+    if (!dbg.arm(1)) return A2SGD_ERR_CUDA;
     return launch_encode(c, grad, grad_stride, err, err_stride, local_means,
                          reinterpret_cast<unsigned long long *>(pos_counts), pos_mask, nullptr,
                          static_cast<cudaStream_t>(stream));
@@ -683,9 +567,12 @@ extern "C" int a2sgd_global_average(a2sgd_ctx *c, const float *local_means, floa
     if (!device_pointer_ok(c, local_means) || !device_pointer_ok(c, global_means)) return A2SGD_ERR_ARG;
     DeviceGuard guard(c->device);
     if (!guard.ok) return A2SGD_ERR_CUDA;
-    k_global_average<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(local_means, c->P, global_means,
-                                                                     c->global_means);
-    A2_CUDA(cudaGetLastError());
+    {
+        uint32_t P = c->P;
+        float *ctx_copy = c->global_means;
+        void *params[] = {&local_means, &P, &global_means, &ctx_copy};
+        A2_CUDA(cudaLaunchKernel(c->k->global_average, dim3(1), dim3(32), params, 0, static_cast<cudaStream_t>(stream)));
+    }
     return A2SGD_OK;
 }
 
@@ -697,9 +584,12 @@ extern "C" int a2sgd_global_average_from_sums(a2sgd_ctx *c, const double *sums, 
     if (!device_pointer_ok(c, sums) || !device_pointer_ok(c, global_means)) return A2SGD_ERR_ARG;
     DeviceGuard guard(c->device);
     if (!guard.ok) return A2SGD_ERR_CUDA;
-    k_global_average_from_sums<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(sums, workers, global_means,
-                                                                                c->global_means);
-    A2_CUDA(cudaGetLastError());
+    {
+        float *ctx_copy = c->global_means;
+        void *params[] = {&sums, &workers, &global_means, &ctx_copy};
+        A2_CUDA(cudaLaunchKernel(c->k->global_average_from_sums, dim3(1), dim3(32), params, 0,
+                                 static_cast<cudaStream_t>(stream)));
+    }
     return A2SGD_OK;
 }
 
@@ -720,6 +610,11 @@ extern "C" int a2sgd_decode_update(a2sgd_ctx *c, float *w, int64_t w_stride, con
         return A2SGD_ERR_ARG;
     DeviceGuard guard(c->device);
     if (!guard.ok) return A2SGD_ERR_CUDA;
+    DebugScope dbg(c, static_cast<cudaStream_t>(stream));
+    dbg.add(grad, c->P, grad_stride, c->n, 4);
+    dbg.add(err, c->P, err_stride, c->n, 4);
+    dbg.add(w, (w_stride == 0 || c->P == 1) ? 1 : c->P, w_stride, c->n, 4);
+    if (!dbg.arm(1)) return A2SGD_ERR_CUDA;
     return launch_decode(c, w, (c->P == 1) ? 0 : w_stride, grad, grad_stride, err, err_stride, local_means,
                          global_means, lr, static_cast<cudaStream_t>(stream));
 }
@@ -737,6 +632,12 @@ extern "C" int a2sgd_step(a2sgd_ctx *c, float *w, int64_t w_stride, const float 
     if (!guard.ok) return A2SGD_ERR_CUDA;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const int64_t ws = (c->P == 1) ? 0 : w_stride;
+    DebugScope dbg(c, s);
+    dbg.add(grad, c->P, grad_stride, c->n, 4);
+    dbg.add(err, c->P, err_stride, c->n, 4);
+    dbg.add(w, ws == 0 ? 1 : c->P, ws, c->n, 4);
+    dbg.add(c->sign_mask, c->P, (int64_t)((c->n + 31) / 32), (c->n + 31) / 32, 4);
+    if (!dbg.arm(1)) return A2SGD_ERR_CUDA;
     if (c->flags & A2SGD_DEFERRED_RESIDUAL) return deferred_step(c, w, ws, grad, grad_stride, err, err_stride, lr, s);
     if (!(c->flags & A2SGD_FORCE_TWO_PASS)) {
         const bool store = !c->alg1 || err != nullptr;
@@ -787,6 +688,12 @@ extern "C" int a2sgd_decode_update_momentum(a2sgd_ctx *c, float *w, int64_t w_st
     mo.mom_stride = mom_stride;
     mo.beta = beta;
     mo.weight_decay = weight_decay;
+    DebugScope dbg(c, static_cast<cudaStream_t>(stream));
+    dbg.add(grad, c->P, grad_stride, c->n, 4);
+    dbg.add(err, c->P, err_stride, c->n, 4);
+    dbg.add(w, (w_stride == 0 || c->P == 1) ? 1 : c->P, w_stride, c->n, 4);
+    dbg.add(mom, (w_stride == 0 || c->P == 1) ? 1 : c->P, mom_stride, c->n, 4);
+    if (!dbg.arm(1)) return A2SGD_ERR_CUDA;
     return launch_decode(c, w, (c->P == 1) ? 0 : w_stride, grad, grad_stride, err, err_stride, local_means,
                          global_means, lr, static_cast<cudaStream_t>(stream), &mo);
 }
@@ -808,6 +715,12 @@ extern "C" int a2sgd_step_momentum(a2sgd_ctx *c, float *w, int64_t w_stride, flo
     mo.mom_stride = mom_stride;
     mo.beta = beta;
     mo.weight_decay = weight_decay;
+    DebugScope dbg(c, s);
+    dbg.add(grad, c->P, grad_stride, c->n, 4);
+    dbg.add(err, c->P, err_stride, c->n, 4);
+    dbg.add(w, (w_stride == 0 || c->P == 1) ? 1 : c->P, w_stride, c->n, 4);
+    dbg.add(mom, (w_stride == 0 || c->P == 1) ? 1 : c->P, mom_stride, c->n, 4);
+    if (!dbg.arm(1)) return A2SGD_ERR_CUDA;
     const int r1 = launch_encode(c, grad, grad_stride, err, err_stride, c->local_means, c->pos_counts, nullptr,
                                  c->global_means, s);
     if (r1) return r1;
@@ -846,6 +759,12 @@ static int step_lowp(a2sgd_ctx *c, float *w, int64_t w_stride, const uint16_t *g
     const bool store = ef || err != nullptr;
     const int64_t ws = (c->P == 1) ? 0 : w_stride;
     const float *g = reinterpret_cast<const float *>(grad); // element type is carried by the kernel template
+    if (!device_pointer_ok(c, grad) || !device_pointer_ok(c, err) || !device_pointer_ok(c, w)) return A2SGD_ERR_ARG;
+    DebugScope dbg(c, s);
+    dbg.add(grad, c->P, grad_stride, c->n, 2);
+    dbg.add(err, c->P, err_stride, c->n, 4);
+    dbg.add(w, ws == 0 ? 1 : c->P, ws, c->n, 4);
+    if (!dbg.arm(1)) return A2SGD_ERR_CUDA;
     int vw_enc = vec_width_bf16(grad, grad_stride, c->P);
     if (ef && vec_width(err, err_stride, c->P) < 8) vw_enc = 0;
     int vw_dec = vw_enc;
@@ -853,7 +772,7 @@ static int step_lowp(a2sgd_ctx *c, float *w, int64_t w_stride, const uint16_t *g
     {
         EncodeArgs a = make_encode_args(c, g, grad_stride, err, err_stride, c->local_means, c->pos_counts, nullptr,
                                         c->global_means);
-        const void *fn = gt == 1 ? select_encode_lowp<1>(ef, vw_enc) : select_encode_lowp<2>(ef, vw_enc);
+        const void *fn = c->k->encode_lowp(gt, ef, vw_enc);
         const uint64_t items = vw_enc ? (c->n + 7) / 8 : (c->n + kScalarU - 1) / kScalarU;
         const dim3 grid(std::min(per_worker_grid(c, occupancy(c, fn), items, kWavesK1), c->g_alloc), c->P);
         void *params[] = {&a};
@@ -861,8 +780,7 @@ static int step_lowp(a2sgd_ctx *c, float *w, int64_t w_stride, const uint16_t *g
     }
     {
         DecodeArgs a = make_decode_args(c, w, ws, g, grad_stride, err, err_stride, c->local_means, c->global_means, lr);
-        const void *fn = gt == 1 ? select_decode_lowp<1>(ef, store, ws == 0, c->P, vw_dec)
-                                 : select_decode_lowp<2>(ef, store, ws == 0, c->P, vw_dec);
+        const void *fn = c->k->decode_lowp(gt, ef, store, ws == 0, c->P, vw_dec);
         const uint64_t items = vw_dec ? (c->n + 7) / 8 : (c->n + kDecScalarU - 1) / kDecScalarU;
         const dim3 grid = (ws == 0) ? dim3(flat_grid(c, occupancy(c, fn), items, kWavesK3))
                                     : dim3(per_worker_grid(c, occupancy(c, fn), items, kWavesK3), c->P);
@@ -881,10 +799,18 @@ extern "C" int a2sgd_materialize_err(a2sgd_ctx *c, float *err, int64_t err_strid
     if (!c->err_holds_v) return A2SGD_OK; // already a true residual
     DeviceGuard guard(c->device);
     if (!guard.ok) return A2SGD_ERR_CUDA;
+    if (!device_pointer_ok(c, err)) return A2SGD_ERR_ARG;
+    DebugScope dbg(c, static_cast<cudaStream_t>(stream));
+    dbg.add(err, c->P, err_stride, c->n, 4);
+    if (!dbg.arm(1)) return A2SGD_ERR_CUDA;
     const uint64_t need = std::max<uint64_t>(1, (c->n / 8 + kBlock - 1) / kBlock);
     const dim3 grid((unsigned)std::min<uint64_t>(need, 0x7fffffffu), c->P);
-    k_materialize_err<<<grid, kBlock, 0, static_cast<cudaStream_t>(stream)>>>(err, err_stride, c->n, c->global_means);
-    A2_CUDA(cudaGetLastError());
+    {
+        uint64_t n = c->n;
+        const float *means = c->global_means;
+        void *params[] = {&err, &err_stride, &n, &means};
+        A2_CUDA(cudaLaunchKernel(c->k->materialize_err, grid, dim3(kBlock), params, 0, static_cast<cudaStream_t>(stream)));
+    }
     c->err_holds_v = false;
     return A2SGD_OK;
 }
@@ -918,6 +844,10 @@ static int dense_sync_impl(a2sgd_ctx *c, float *w, int64_t w_stride, const float
     if (!guard.ok) return A2SGD_ERR_CUDA;
     const int64_t ws = (c->P == 1) ? 0 : w_stride;
     const int vw = std::min(vec_width(grad, grad_stride, c->P), vec_width(w, ws == 0 ? 8 : ws, c->P));
+    DebugScope dbg(c, static_cast<cudaStream_t>(stream));
+    dbg.add(grad, c->P, grad_stride, c->n, 4);
+    dbg.add(w, ws == 0 ? 1 : c->P, ws, c->n, 4);
+    if (!dbg.arm(1)) return A2SGD_ERR_CUDA;
     DenseArgs a{};
     a.w = w;
     a.w_stride = ws;
@@ -927,7 +857,7 @@ static int dense_sync_impl(a2sgd_ctx *c, float *w, int64_t w_stride, const float
     a.P = c->P;
     a.lr = lr;
     a.divisor = divisor;
-    const void *fn = select_dense(c->P, vw, ws != 0);
+    const void *fn = c->k->dense(c->P, vw, ws != 0);
     const uint64_t items = vw ? (c->n + vw - 1) / vw : c->n;
     const dim3 grid(flat_grid(c, occupancy(c, fn), items, kWavesK3));
     void *params[] = {&a};
@@ -936,18 +866,6 @@ static int dense_sync_impl(a2sgd_ctx *c, float *w, int64_t w_stride, const float
 }
 
 // ---------------------------------------------------------------- segment lists
-template <bool EF, bool STORE>
-const void *select_decode_segments_p(uint32_t P)
-{
-    switch (P) {
-    case 1: return (const void *)k_decode_segments<EF, STORE, 1>;
-    case 2: return (const void *)k_decode_segments<EF, STORE, 2>;
-    case 4: return (const void *)k_decode_segments<EF, STORE, 4>;
-    case 8: return (const void *)k_decode_segments<EF, STORE, 8>;
-    default: return (const void *)k_decode_segments<EF, STORE, 0>;
-    }
-}
-
 extern "C" int a2sgd_segments_create(a2sgd_ctx *c, uint32_t S, const uint64_t *numel, const float *const *grad,
                                      float *const *err, float *const *w, int w_replicated, a2sgd_segments **out)
 {
@@ -968,14 +886,15 @@ extern "C" int a2sgd_segments_create(a2sgd_ctx *c, uint32_t S, const uint64_t *n
         for (uint32_t p = 0; p < P; ++p) {
             const float *g = grad[(size_t)p * S + s];
             const float *e = err ? err[(size_t)p * S + s] : nullptr;
-            if (!g || (!c->alg1 && !e)) return A2SGD_ERR_ARG;
+            if (!g || (err && !e)) return A2SGD_ERR_ARG; // an error table, when given, has no NULL entries
+            if (!device_pointer_ok(c, g) || !device_pointer_ok(c, e)) return A2SGD_ERR_ARG;
             if (!aligned(g, 4) || (e && !aligned(e, 4))) return A2SGD_ERR_ALIGN;
             vec = vec && aligned(g, 32) && (!e || aligned(e, 32));
         }
         const uint32_t w_rows = repl ? P : 1;
         for (uint32_t r = 0; r < w_rows; ++r) {
             const float *wp = w[(size_t)r * S + s];
-            if (!wp) return A2SGD_ERR_ARG;
+            if (!wp || !device_pointer_ok(c, wp)) return A2SGD_ERR_ARG;
             if (!aligned(wp, 4)) return A2SGD_ERR_ALIGN;
             vec = vec && aligned(wp, 32);
         }
@@ -1054,7 +973,7 @@ static int launch_encode_segments(a2sgd_ctx *c, a2sgd_segments *sg, float *local
 {
     SegTables t = seg_tables(sg, nullptr);
     EncodeArgs a = make_encode_args(c, nullptr, 0, nullptr, 0, local_means, pos_counts, nullptr, global_means);
-    const void *fn = !c->alg1 ? (const void *)k_encode_segments<true> : (const void *)k_encode_segments<false>;
+    const void *fn = c->k->encode_segments(!c->alg1);
     const uint64_t slots = (uint64_t)c->sm_count * occupancy(c, fn) * kWavesK1;
     uint64_t G = std::max<uint64_t>(1, slots / c->P);
     G = std::min<uint64_t>(std::min<uint64_t>(G, sg->n_tiles), c->g_alloc);
@@ -1071,9 +990,7 @@ static int launch_decode_segments(a2sgd_ctx *c, a2sgd_segments *sg, const float 
     SegTables t = seg_tables(sg, lr_per_segment);
     DecodeArgs a = make_decode_args(c, nullptr, sg->replicated ? 1 : 0, nullptr, 0, nullptr, 0, local_means,
                                     global_means, lr);
-    const void *fn = ef ? select_decode_segments_p<true, true>(c->P)
-                        : store ? select_decode_segments_p<false, true>(c->P)
-                                : select_decode_segments_p<false, false>(c->P);
+    const void *fn = c->k->decode_segments(ef, store, c->P);
     const uint64_t grid = std::min<uint64_t>(sg->n_tiles, 0x7fffffffu);
     void *params[] = {&a, &t};
     A2_CUDA(launch_pdl(fn, dim3((unsigned)grid), params, s));
@@ -1087,6 +1004,8 @@ static int step_segments_impl(a2sgd_ctx *c, a2sgd_segments *sg, float lr, const 
     DeviceGuard guard(c->device);
     if (!guard.ok) return A2SGD_ERR_CUDA;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
+    DebugScope dbg(c, s);
+    if (!dbg.arm(2)) return A2SGD_ERR_CUDA;
     const int rc = launch_encode_segments(c, sg, c->local_means, c->pos_counts, c->global_means, s);
     if (rc) return rc;
     return launch_decode_segments(c, sg, c->local_means, c->global_means, lr, lr_per_segment, s);
@@ -1111,6 +1030,8 @@ extern "C" int a2sgd_encode_segments(a2sgd_ctx *c, a2sgd_segments *sg, float *lo
     if (!device_pointer_ok(c, local_means) || !device_pointer_ok(c, pos_counts)) return A2SGD_ERR_ARG;
     DeviceGuard guard(c->device);
     if (!guard.ok) return A2SGD_ERR_CUDA;
+    DebugScope dbg(c, static_cast<cudaStream_t>(stream));
+    if (!dbg.arm(2)) return A2SGD_ERR_CUDA;
     return launch_encode_segments(c, sg, local_means, reinterpret_cast<unsigned long long *>(pos_counts), nullptr,
                                   static_cast<cudaStream_t>(stream));
 }
@@ -1129,6 +1050,8 @@ extern "C" int a2sgd_decode_update_segments(a2sgd_ctx *c, a2sgd_segments *sg, co
         return A2SGD_ERR_ARG;
     DeviceGuard guard(c->device);
     if (!guard.ok) return A2SGD_ERR_CUDA;
+    DebugScope dbg(c, static_cast<cudaStream_t>(stream));
+    if (!dbg.arm(2)) return A2SGD_ERR_CUDA;
     return launch_decode_segments(c, sg, local_means, global_means, lr, lr_per_segment,
                                   static_cast<cudaStream_t>(stream));
 }
@@ -1195,10 +1118,10 @@ extern "C" int a2sgd_launch_info(a2sgd_ctx *c, int64_t w_stride, uint32_t out[5]
     const bool shared = w_stride == 0 || c->P == 1;
     const int vw = kMaxVecWidth >= 8 ? 8 : 4;
     const uint64_t items = (c->n + vw - 1) / vw;
-    out[0] = std::min(per_worker_grid(c, occupancy(c, select_encode(ef, false, vw)), items, kWavesK1),
+    out[0] = std::min(per_worker_grid(c, occupancy(c, c->k->encode(ef, false, vw)), items, kWavesK1),
                       c->g_alloc) * c->P;
-    out[1] = shared ? flat_grid(c, occupancy(c, select_decode_shared(ef, true, c->P, vw)), items, kWavesK3)
-                    : per_worker_grid(c, occupancy(c, select_decode_repl(ef, true, vw)), items, kWavesK3) * c->P;
+    out[1] = shared ? flat_grid(c, occupancy(c, c->k->decode_shared(ef, true, c->P, vw, false)), items, kWavesK3)
+                    : per_worker_grid(c, occupancy(c, c->k->decode_repl(ef, true, vw, false)), items, kWavesK3) * c->P;
     out[2] = kBlock;
     out[3] = 0;
     if (!(c->flags & A2SGD_FORCE_TWO_PASS)) {
@@ -1223,6 +1146,7 @@ extern "C" const char *a2sgd_status_string(int status)
     case A2SGD_ERR_NONFINITE: return "non-finite group sum";
     case A2SGD_ERR_NOMEM: return "scratch allocation failed";
     case A2SGD_ERR_TOO_LARGE: return "too large: n*P for the single-launch path, or P for the fixed scratch";
+    case A2SGD_ERR_BOUNDS: return "debug checks: an access outside the buffers of the call was skipped";
     default: return "unknown status";
     }
 }

@@ -24,13 +24,27 @@
 // integers.  No floating-point atomics: each CTA stores one partial, and the
 // CTA that draws the last ticket folds all partials in index order, so the
 // result depends only on (n, P, grid), never on scheduling.
-#pragma once
-
+//
+// This header is compiled twice into the library, into two namespaces: the production kernels
+// (A2SGD_NS = a2sgd, A2SGD_CHECKED = 0) and a checked copy of exactly the same code
+// (a2sgd_chk, A2SGD_CHECKED = 1) in which every access made through the helpers below is first
+// tested against the extents of the call's buffers (A2SGD_DEBUG_CHECKS).  Keeping the two apart
+// at compile time leaves the production kernels' instructions and register counts untouched.
+// No include guard: the including file sets the two macros.
 #include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
-namespace a2sgd {
+#include "a2sgd_debug_check.h"
+
+#ifndef A2SGD_NS
+#define A2SGD_NS a2sgd
+#endif
+#ifndef A2SGD_CHECKED
+#define A2SGD_CHECKED 0
+#endif
+
+namespace A2SGD_NS {
 
 constexpr int kBlock = 256;
 constexpr int kWarps = kBlock / 32;
@@ -41,6 +55,51 @@ constexpr int kMaxP = 1024;
 constexpr int kDevOk = 0;
 constexpr int kDevTimeout = -4;
 constexpr int kDevNonFinite = -5;
+constexpr int kDevBounds = -8;
+
+// ------------------------------------------------------------------ A2SGD_DEBUG_CHECKS
+// The stand-in for a memory checker on systems where none can be run.  In the checked copy of
+// the kernels, while the descriptor below is switched on (by a context created with
+// A2SGD_DEBUG_CHECKS, for the duration of its launches), every access that goes through the
+// helpers of this file is first checked against the extents of the buffers the call was given
+// — inside the live elements of one row of one buffer — and an access that is not is SKIPPED
+// (loads return 0) and latches kDevBounds in the context's status word.  Nothing traps, so a
+// defect shows up as a status code instead of a fault.  One descriptor per device: launches of a
+// checking context must not overlap other checked launches on the same device.
+using a2sgd_check::DebugRange;
+using a2sgd_check::kDebugMaxRanges;
+struct DebugChecks {
+    int on;    // 0 off, 1 address ranges below, 2 index checks only (the tensors of a segment list)
+    int count;
+    int *status;
+    DebugRange range[kDebugMaxRanges];
+};
+#if A2SGD_CHECKED
+static __constant__ DebugChecks c_debug;
+
+static __device__ __noinline__ bool debug_access_failed(const void *p, unsigned bytes)
+{
+    if (a2sgd_check::debug_any_range_contains(c_debug.range, c_debug.count, (uint64_t)(uintptr_t)p, bytes)) return false;
+    atomicCAS(c_debug.status, kDevOk, kDevBounds);
+    return true;
+}
+// true: the access may be made
+__device__ __forceinline__ bool access_ok(const void *p, unsigned bytes)
+{
+    if (c_debug.on != 1) return true;
+    return !debug_access_failed(p, bytes);
+}
+// the index form, for the tensors of a segment list
+__device__ __forceinline__ bool span_ok(uint64_t first, uint64_t count, uint64_t numel)
+{
+    if (c_debug.on == 0 || a2sgd_check::debug_span_inside(first, count, numel)) return true;
+    atomicCAS(c_debug.status, kDevOk, kDevBounds);
+    return false;
+}
+#else
+__device__ __forceinline__ bool access_ok(const void *, unsigned) { return true; }
+__device__ __forceinline__ bool span_ok(uint64_t, uint64_t, uint64_t) { return true; }
+#endif
 
 struct __align__(8) Partial {
     double s_pos;
@@ -80,6 +139,10 @@ template <>
 __device__ __forceinline__ Vec<4> ld_vec<4>(const float *p)
 {
     Vec<4> r;
+    if (!access_ok(p, 16)) {
+        r.v[0] = r.v[1] = r.v[2] = r.v[3] = 0.f;
+        return r;
+    }
     asm volatile("ld.global.L1::no_allocate.v4.f32 {%0,%1,%2,%3}, [%4];"
                  : "=f"(r.v[0]), "=f"(r.v[1]), "=f"(r.v[2]), "=f"(r.v[3])
                  : "l"(p));
@@ -89,6 +152,11 @@ template <>
 __device__ __forceinline__ Vec<8> ld_vec<8>(const float *p)
 {
     Vec<8> r;
+    if (!access_ok(p, 32)) {
+#pragma unroll
+        for (int k = 0; k < 8; ++k) r.v[k] = 0.f;
+        return r;
+    }
     asm volatile("ld.global.L1::no_allocate.L2::evict_first.v8.f32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
                  : "=f"(r.v[0]), "=f"(r.v[1]), "=f"(r.v[2]), "=f"(r.v[3]), "=f"(r.v[4]), "=f"(r.v[5]),
                    "=f"(r.v[6]), "=f"(r.v[7])
@@ -100,6 +168,7 @@ __device__ __forceinline__ void st_vec(float *p, const Vec<VW> &x);
 template <>
 __device__ __forceinline__ void st_vec<4>(float *p, const Vec<4> &x)
 {
+    if (!access_ok(p, 16)) return;
     asm volatile("st.global.L1::no_allocate.v4.f32 [%0], {%1,%2,%3,%4};" ::"l"(p), "f"(x.v[0]), "f"(x.v[1]),
                  "f"(x.v[2]), "f"(x.v[3])
                  : "memory");
@@ -107,6 +176,7 @@ __device__ __forceinline__ void st_vec<4>(float *p, const Vec<4> &x)
 template <>
 __device__ __forceinline__ void st_vec<8>(float *p, const Vec<8> &x)
 {
+    if (!access_ok(p, 32)) return;
     asm volatile("st.global.L1::no_allocate.L2::evict_first.v8.f32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(p),
                  "f"(x.v[0]), "f"(x.v[1]), "f"(x.v[2]), "f"(x.v[3]), "f"(x.v[4]), "f"(x.v[5]), "f"(x.v[6]),
                  "f"(x.v[7])
@@ -115,16 +185,29 @@ __device__ __forceinline__ void st_vec<8>(float *p, const Vec<8> &x)
 __device__ __forceinline__ float ld_stream1(const float *p)
 {
     float r;
+    if (!access_ok(p, 4)) return 0.f;
     asm volatile("ld.global.L1::no_allocate.f32 %0, [%1];" : "=f"(r) : "l"(p));
     return r;
 }
 __device__ __forceinline__ void st_stream1(float *p, float v)
 {
+    if (!access_ok(p, 4)) return;
     asm volatile("st.global.L1::no_allocate.f32 [%0], %1;" ::"l"(p), "f"(v) : "memory");
 }
 
-// A gradient row whose elements are fp32 (GB = 0), bfloat16 (GB = 1) or IEEE half (GB = 2); the
-// paper notes that the method "can be further integrated with quantization".  Widening either
+// Plain (cached) single-element accesses: the read-modify-write tails and the mask words.
+__device__ __forceinline__ float ld1(const float *p) { return access_ok(p, 4) ? *p : 0.f; }
+__device__ __forceinline__ void st1(float *p, float v)
+{
+    if (access_ok(p, 4)) *p = v;
+}
+__device__ __forceinline__ void st_word(uint32_t *p, uint32_t v)
+{
+    if (access_ok(p, 4)) *p = v;
+}
+
+// A gradient row whose elements are fp32 (GB = 0), bfloat16 (GB = 1) or IEEE half (GB = 2);
+// Section 1 of the paper names the combination with quantisation as a natural extension.  Widening either
 // 16-bit format to fp32 is exact (bfloat16 is the upper half of an fp32; every half value,
 // subnormals included, is an fp32 value), so v = float(g) + e is formed from exactly the value the
 // caller stored.
@@ -138,8 +221,9 @@ struct GradRow {
     __device__ __forceinline__ float one(uint64_t elem) const
     {
         if (GB) {
-            unsigned short h;
-            asm volatile("ld.global.L1::no_allocate.u16 %0, [%1];" : "=h"(h) : "l"(base + 2 * elem));
+            unsigned short h = 0;
+            if (access_ok(base + 2 * elem, 2))
+                asm volatile("ld.global.L1::no_allocate.u16 %0, [%1];" : "=h"(h) : "l"(base + 2 * elem));
             return GB == 1 ? __uint_as_float((unsigned)h << 16) : __half2float(__ushort_as_half(h));
         }
         return ld_stream1(reinterpret_cast<const float *>(base) + elem);
@@ -149,10 +233,11 @@ struct GradRow {
     {
         if (GB) {
             static_assert(!GB || VW == 8, "16-bit gradients use 8-element (128-bit) vectors");
-            unsigned x[4];
-            asm volatile("ld.global.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
-                         : "=r"(x[0]), "=r"(x[1]), "=r"(x[2]), "=r"(x[3])
-                         : "l"(base + 2 * elem));
+            unsigned x[4] = {0u, 0u, 0u, 0u};
+            if (access_ok(base + 2 * elem, 16))
+                asm volatile("ld.global.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                             : "=r"(x[0]), "=r"(x[1]), "=r"(x[2]), "=r"(x[3])
+                             : "l"(base + 2 * elem));
             Vec<VW> r;
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
@@ -435,7 +520,7 @@ __global__ void __launch_bounds__(kBlock) k_encode_vec(EncodeArgs a)
 #pragma unroll
             for (int x = 1; x < LPW; x <<= 1) w |= __shfl_xor_sync(group_mask, w, x);
             const uint64_t word = jv / LPW;
-            if (sub == 0 && word < full_words) mask[word] = w;
+            if (sub == 0 && word < full_words) st_word(mask + word, w);
         }
     };
 
@@ -499,7 +584,7 @@ __global__ void __launch_bounds__(kBlock) k_encode_vec(EncodeArgs a)
                 pos = v >= 0.0f;
             }
             const unsigned w = __ballot_sync(0xffffffffu, pos);
-            if (lane == 0) mask[full_words] = w;
+            if (lane == 0) st_word(mask + full_words, w);
         }
     }
     double s_pos = acc.s_pos, s_neg = acc.s_neg;
@@ -563,7 +648,7 @@ __global__ void __launch_bounds__(kBlock) k_encode_scalar(EncodeArgs a)
             if (whole || i < a.n) split1(v, sp[k], sn[k], acc.n_pos, bit);
             if (MASK && (whole || (i - lane) < a.n)) {       // warp-uniform: the warp's 32 elements share a word
                 const unsigned w = __ballot_sync(0xffffffffu, bit != 0);
-                if (lane == 0) mask[i >> 5] = w;
+                if (lane == 0) st_word(mask + (i >> 5), w);
             }
         }
         acc.s_pos += (double)tree_sum<kScalarU>(sp);
@@ -827,9 +912,9 @@ __global__ void __launch_bounds__(kBlock) k_decode_shared_vec(DecodeArgs a)
                 sum += gh;
                 if (STORE) st_stream1(a.err + (int64_t)p * a.err_stride + i, rs);
             }
-            float m = MOM ? a.mom[i] : 0.f;
-            a.w[i] = update1<MOM>(uc, sum, a.w[i], m);
-            if (MOM) a.mom[i] = m;
+            float m = MOM ? ld1(a.mom + i) : 0.f;
+            st1(a.w + i, update1<MOM>(uc, sum, ld1(a.w + i), m));
+            if (MOM) st1(a.mom + i, m);
         }
     }
 }
@@ -894,9 +979,9 @@ __global__ void __launch_bounds__(kBlock) k_decode_repl_vec(DecodeArgs a)
             float gh, rs;
             decode1<EF>(v, c, gh, rs);
             if (STORE) st_stream1(e + i, rs);
-            float m = MOM ? mom[i] : 0.f;
-            w[i] = update1<MOM>(uc, gh, w[i], m);
-            if (MOM) mom[i] = m;
+            float m = MOM ? ld1(mom + i) : 0.f;
+            st1(w + i, update1<MOM>(uc, gh, ld1(w + i), m));
+            if (MOM) st1(mom + i, m);
         }
     }
 }
@@ -1058,15 +1143,15 @@ __global__ void __launch_bounds__(kBlock) k_decode_deferred(DeferredDecodeArgs a
         if (i < a.n) {
             float sum = 0.f;
             for (uint32_t p = 0; p < P; ++p) {
-                const float gh = (__ldcg(a.v + (int64_t)p * a.v_stride + i) >= 0.0f) ? g_pos : g_neg;
+                const float gh = (ld1(a.v + (int64_t)p * a.v_stride + i) >= 0.0f) ? g_pos : g_neg;
                 if (REPL) {
                     float *wp = a.w + (int64_t)p * a.w_stride + i;
-                    *wp = fmaf(scale, gh, *wp);
+                    st1(wp, fmaf(scale, gh, ld1(wp)));
                 } else {
                     sum += gh;
                 }
             }
-            if (!REPL) a.w[i] = fmaf(scale, sum, a.w[i]);
+            if (!REPL) st1(a.w + i, fmaf(scale, sum, ld1(a.w + i)));
         }
     }
 }
@@ -1089,7 +1174,10 @@ static __global__ void __launch_bounds__(kBlock) k_materialize_err(float *v, int
     }
     if (blockIdx.x == 0 && threadIdx.x < 8) {
         const uint64_t i = nv * 8 + threadIdx.x;
-        if (i < n) row[i] = row[i] - (row[i] >= 0.0f ? g_pos : g_neg);
+        if (i < n) {
+            const float x = ld1(row + i);
+            st1(row + i, x - (x >= 0.0f ? g_pos : g_neg));
+        }
     }
 }
 
@@ -1147,7 +1235,7 @@ __global__ void __launch_bounds__(kBlock) k_dense_sync_vec(DenseArgs a)
             const uint32_t reps = REPL ? P : 1;
             for (uint32_t r = 0; r < reps; ++r) {
                 float *wp = a.w + (int64_t)r * a.w_stride + i;
-                *wp = fmaf(scale, sum, *wp);
+                st1(wp, fmaf(scale, sum, ld1(wp)));
             }
         }
     }
@@ -1166,7 +1254,7 @@ __global__ void __launch_bounds__(kBlock) static k_dense_sync_scalar(DenseArgs a
         for (uint32_t p = 0; p < a.P; ++p) sum += ld_stream1(a.grad + (int64_t)p * a.grad_stride + i);
         for (uint32_t r = 0; r < reps; ++r) {
             float *wp = a.w + (int64_t)r * a.w_stride + i;
-            *wp = fmaf(scale, sum, *wp);
+            st1(wp, fmaf(scale, sum, ld1(wp)));
         }
     }
 }
@@ -1474,10 +1562,10 @@ __global__ void __launch_bounds__(kBlock) k_step_coop(CoopArgs a)
                 sum += gh;
             } else {
                 float *wp = da.w + (int64_t)p * da.w_stride + i_tail;
-                *wp = fmaf(scale, gh, *wp);
+                st1(wp, fmaf(scale, gh, ld1(wp)));
             }
         }
-        if (SHARED) da.w[i_tail] = fmaf(scale, sum, da.w[i_tail]);
+        if (SHARED) st1(da.w + i_tail, fmaf(scale, sum, ld1(da.w + i_tail)));
     }
 }
 
@@ -1570,11 +1658,11 @@ __global__ void __launch_bounds__(kBlock) k_step_coop_l2(CoopArgs a)
                 sum += gh;
             } else {
                 float *wp = da.w + (int64_t)p * da.w_stride + i_tail;
-                *wp = fmaf(scale, gh, *wp);
+                st1(wp, fmaf(scale, gh, ld1(wp)));
             }
         }
-        if (SHARED) da.w[i_tail] = fmaf(scale, sum, da.w[i_tail]);
+        if (SHARED) st1(da.w + i_tail, fmaf(scale, sum, ld1(da.w + i_tail)));
     }
 }
 
-} // namespace a2sgd
+} // namespace A2SGD_NS

@@ -23,6 +23,8 @@
 #include <cstdint>
 #include <mutex>
 
+#define A2SGD_NS a2sgd
+#define A2SGD_CHECKED 0
 #include "a2sgd_kernels.cuh"
 
 using namespace a2sgd;

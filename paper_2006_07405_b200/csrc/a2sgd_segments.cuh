@@ -1,8 +1,8 @@
 // Segment-list (multi-tensor) forms of K1 and K3: the model is a list of
 // tensors living in separate allocations, as a training framework holds them,
-// and is reduced to the same two whole-model means per worker ("for each
-// model, it traverses all gradients to compute two separate averages",
-// Section 4.3) without first being copied into one flat vector.
+// and is reduced to the same two whole-model means per worker (Section 4.3:
+// the two averages are taken over all gradients of the model) without first
+// being copied into one flat vector.
 //
 // The flat index space of each tensor is cut into tiles of kSegTile elements;
 // a table built once per plan maps tile -> (tensor, offset).  A tile never
@@ -10,11 +10,9 @@
 // pointer plus a contiguous range.  Tensors whose pointers are all 32-byte
 // aligned take 256-bit accesses; any other 4-byte alignment takes coalesced
 // scalar accesses (decided per tensor on the host, uniform per CTA).
-#pragma once
-
-#include "a2sgd_kernels.cuh"
-
-namespace a2sgd {
+// Like a2sgd_kernels.cuh this header has no include guard: it is compiled once per kernel variant,
+// after a2sgd_kernels.cuh, into the namespace A2SGD_NS.
+namespace A2SGD_NS {
 
 constexpr int kSegVW = 8;
 constexpr uint32_t kSegTile = kBlock * kSegVW; // 2048 elements per tile
@@ -72,7 +70,12 @@ __global__ void __launch_bounds__(kBlock) k_encode_segments(EncodeArgs a, SegTab
     Acc acc;
     for (uint64_t tile = blockIdx.x; tile < t.n_tiles; tile += gridDim.x) {
         const SegTile d = t.tiles[tile];
+        if (d.seg >= t.S) {                     // only reachable with a corrupt table
+            span_ok(d.seg, 1, t.S);
+            continue;
+        }
         const uint64_t n_s = t.numel[d.seg];
+        if (!span_ok(d.offset, 1, n_s)) continue;
         const float *__restrict__ g = t.grad[(uint64_t)p * t.S + d.seg];
         const float *__restrict__ e = EF ? t.err[(uint64_t)p * t.S + d.seg] : nullptr;
         float sp = 0.f, sn = 0.f;
@@ -157,6 +160,7 @@ __global__ void __launch_bounds__(kBlock) k_decode_segments(DecodeArgs a, SegTab
             d = t.tiles[tile];
             n_s = __ldg(t.numel + d.seg);
         }
+        if (!span_ok(d.offset, 1, n_s)) continue; // the tile starts inside its tensor
         const uint64_t i = d.offset + (uint64_t)threadIdx.x * kSegVW;
         // layer-wise learning rates (e.g. LARS, which the paper uses for VGG-16): one per tensor
         const float lr = t.lr_per_segment ? __ldg(t.lr_per_segment + d.seg) : a.lr;
@@ -237,18 +241,18 @@ __global__ void __launch_bounds__(kBlock) k_decode_segments(DecodeArgs a, SegTab
                     if (STORE) st_stream1(t.err[(uint64_t)p * t.S + d.seg] + idx, rs);
                     if (repl) {
                         float *wp = t.w[(uint64_t)p * t.S + d.seg] + idx;
-                        *wp = fmaf(scale, gh, *wp);
+                        st1(wp, fmaf(scale, gh, ld1(wp)));
                     } else {
                         sum += gh;
                     }
                 }
                 if (!repl) {
                     float *wp = t.w[d.seg] + idx;
-                    *wp = fmaf(scale, sum, *wp);
+                    st1(wp, fmaf(scale, sum, ld1(wp)));
                 }
             }
         }
     }
 }
 
-} // namespace a2sgd
+} // namespace A2SGD_NS

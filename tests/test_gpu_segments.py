@@ -157,3 +157,76 @@ def test_per_segment_learning_rates(mode, replicated):
     assert_state(w_got, wh, _cat(err), eh, gm_ref, "per-segment lr")
     plan.destroy()
     ctx.destroy()
+
+
+@pytest.mark.parametrize("mode", [EF, ALG1])
+def test_staged_segment_calls_match_oracle(mode):
+    """a2sgd_encode_segments -> a2sgd_global_average -> a2sgd_decode_update_segments, the three
+    stages as separate calls on caller-owned means, against the oracle on the concatenation."""
+    P = 3
+    sizes = [2048, 5, 70_001, 4096, 999]
+    n = sum(sizes)
+    gen = torch.Generator("cuda").manual_seed(5)
+    grad = [_tensors(sizes, [0, 1], gen, 1e-3) for _ in range(P)]
+    err = [_tensors(sizes, [0, 1], gen, 3e-4) for _ in range(P)]
+    w = _tensors(sizes, [0, 1], gen, 0.02)
+    gh, eh, wh = _cat(grad), _cat(err), _cat([w])[0]
+    ctx = B.a2sgd_create(n, P, 0, mode)
+    plan = B.a2sgd_segments_create(ctx, grad, err, w)
+    lm = torch.full((P + 2, 2), float("nan"), device="cuda")
+    cnt = torch.zeros(P, dtype=torch.int64, device="cuda")
+    gm = torch.zeros(2, device="cuda")
+    B.a2sgd_encode_segments(ctx, plan, lm[1:P + 1], cnt)
+    B.a2sgd_global_average(ctx, lm[1:P + 1], gm)
+    B.a2sgd_decode_update_segments(ctx, plan, lm[1:P + 1], gm, 0.1)
+    lm_ref, gm_ref, cnt_ref = oracle.step(wh, gh, eh, 0.1, mode=mode)
+    assert np.array_equal(cnt.cpu().numpy().astype(np.uint64), cnt_ref)
+    assert_means(lm[1:P + 1].cpu().numpy(), lm_ref)
+    assert_means(gm.cpu().numpy(), gm_ref)
+    assert torch.isnan(lm[0]).all() and torch.isnan(lm[P + 1]).all()      # two floats per worker, nothing else
+    assert_state(_cat([w])[0], wh, _cat(err), eh, gm_ref, "staged segments")
+    plan.destroy()
+    ctx.destroy()
+
+
+def test_thousands_of_tensors_take_the_tile_table_path():
+    """More tensors than the decode kernel scans for (it then reads per-tile descriptors instead)."""
+    P, S = 2, 4500
+    rng = np.random.default_rng(9)
+    sizes = [int(x) for x in rng.integers(1, 40, size=S)] + [5000]
+    n = sum(sizes)
+    gen = torch.Generator("cuda").manual_seed(11)
+    flat_g = torch.empty((P, n), device="cuda").normal_(0, 1e-3, generator=gen)
+    flat_e = torch.empty((P, n), device="cuda").normal_(0, 3e-4, generator=gen)
+    flat_w = torch.empty(n, device="cuda").normal_(0, 0.02, generator=gen)
+    gh, eh, wh = flat_g.cpu().numpy(), flat_e.cpu().numpy(), flat_w.cpu().numpy()
+    grad = [list(torch.split(flat_g[p], sizes)) for p in range(P)]       # views at arbitrary 4-byte offsets
+    err = [list(torch.split(flat_e[p], sizes)) for p in range(P)]
+    w = list(torch.split(flat_w, sizes))
+    ctx = B.a2sgd_create(n, P, 0, EF)
+    plan = B.a2sgd_segments_create(ctx, grad, err, w)
+    B.a2sgd_step_segments(ctx, plan, 0.1)
+    lm, gm, cnt, status = B.a2sgd_read_stats(ctx)
+    lm_ref, gm_ref, cnt_ref = oracle.step(wh, gh, eh, 0.1, mode=oracle.MODE_EF)
+    assert status == B.OK and np.array_equal(cnt, cnt_ref)
+    assert_means(lm, lm_ref)
+    assert_means(gm, gm_ref)
+    assert_state(flat_w.cpu().numpy(), wh, flat_e.cpu().numpy(), eh, gm_ref, "4501 tensors")
+    plan.destroy()
+    ctx.destroy()
+
+
+def test_alg1_error_table_with_a_missing_entry_is_rejected():
+    ctx = B.a2sgd_create(100, 2, 0, ALG1)
+    g = [[torch.zeros(60, device="cuda"), torch.zeros(40, device="cuda")] for _ in range(2)]
+    w = [torch.zeros(60, device="cuda"), torch.zeros(40, device="cuda")]
+    import ctypes
+    numel = (ctypes.c_uint64 * 2)(60, 40)
+    vp = ctypes.c_void_p
+    g_tab = (vp * 4)(*[t.data_ptr() for row in g for t in row])
+    e_tab = (vp * 4)(g[0][0].data_ptr(), None, g[1][0].data_ptr(), g[1][1].data_ptr())   # one NULL entry
+    w_tab = (vp * 2)(*[t.data_ptr() for t in w])
+    out = vp()
+    rc = B.lib().a2sgd_segments_create(ctx.handle, 2, numel, g_tab, e_tab, w_tab, 0, ctypes.byref(out))
+    assert rc == B.ERR_ARG and not out
+    ctx.destroy()
