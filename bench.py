@@ -128,7 +128,7 @@ class ClockSampler:
 
 
 # ----------------------------------------------------------------------------- reference arm
-def oracle_sample_rate(wl, target_seconds: float, gen_device="cpu"):
+def oracle_sample_rate(wl, target_seconds: float, gen_device="cpu", all_cores=False):
     """Times the CPU oracle (single thread, unmodified) on a prefix sample of the workload's
     flat vector: all P workers, the first n_s elements of each.  Returns a dict."""
     import numpy as np
@@ -136,7 +136,8 @@ def oracle_sample_rate(wl, target_seconds: float, gen_device="cpu"):
     import oracle
     from paper_2006_07405_b200 import workloads as W
 
-    def run(n_s, steps=1):
+    def run(n_s, steps=1, fn=None, skip_first=False):
+        fn = fn or oracle.step
         g = torch.empty((wl.P, n_s))
         sub = W.scaled(wl, max(1, wl.n // n_s))
         gfull = torch.empty((wl.P, sub.n))
@@ -146,18 +147,32 @@ def oracle_sample_rate(wl, target_seconds: float, gen_device="cpu"):
         g = g.numpy()
         e = np.zeros_like(g)
         w = np.zeros(n_s, np.float32)
+        if skip_first:
+            fn(w, g, e, wl.lr, mode=oracle.MODE_EF)
+            steps -= 1
         t0 = time.perf_counter()
         for _ in range(steps):
-            oracle.step(w, g, e, wl.lr, mode=oracle.MODE_EF)
+            fn(w, g, e, wl.lr, mode=oracle.MODE_EF)
         return (time.perf_counter() - t0) / steps
 
     probe_n = min(wl.n, 1 << 20)
     t_probe = run(probe_n)
     n_s = int(min(wl.n, max(probe_n, probe_n * target_seconds / max(t_probe, 1e-9))))
     t = run(n_s)
-    return {"value": n_s / t, "unit": UNIT, "cores": 1, "kind": "oracle",
-            "sample": f"first {n_s} of {wl.n} elements of each of the {wl.P} workers, 1 step, {t:.2f} s",
-            "_n_s": n_s, "_seconds": t}
+    out = {"value": n_s / t, "unit": UNIT, "cores": 1, "kind": "oracle",
+           "sample": f"first {n_s} of {wl.n} elements of each of the {wl.P} workers, 1 step, {t:.2f} s",
+           "_n_s": n_s, "_seconds": t}
+    if all_cores:
+        # the same sample through the OpenMP copy of the step (a separate function: the pinned
+        # oracle stays single-threaded); two steps, the second one timed
+        try:
+            threads = oracle.omp_threads()
+            t_all = run(n_s, steps=2, fn=oracle.step_all_cores, skip_first=True)
+            out["all_cores"] = {"value": n_s / t_all, "unit": UNIT, "cores": threads,
+                                "kind": "OpenMP copy of the oracle's step", "seconds": t_all}
+        except Exception as ex:   # no OpenMP runtime on the box: report, do not fail the bench
+            out["all_cores"] = {"unavailable": str(ex)[:200]}
+    return out
 
 
 def run_reference(args):
@@ -204,8 +219,12 @@ def run_variant(wl, variant, steps, warmup, dev):
     from paper_2006_07405_b200 import binding as B
     from paper_2006_07405_b200 import workloads as W
     n, P = wl.n, wl.P
-    g = B.padded_rows(P, n, dev)
-    e = B.padded_rows(P, n, dev, fill=0.0)
+    if variant == "misaligned":      # rows 4-byte aligned only, each at a different phase
+        g = torch.empty((P, n + 1), device=dev)[:, :n]
+        e = torch.zeros((P, n + 1), device=dev)[:, :n]
+    else:
+        g = B.padded_rows(P, n, dev)
+        e = B.padded_rows(P, n, dev, fill=0.0)
     w = torch.empty(n, device=dev)
     W.fill_gradients(wl, 0, g)
     W.init_weights(wl, w)
@@ -221,6 +240,13 @@ def run_variant(wl, variant, steps, warmup, dev):
         g16 = torch.empty((P, g.stride(0)), dtype=torch.bfloat16, device=dev)[:, :n]
         g16.copy_(g)
         call = lambda: B.a2sgd_step_bf16(ctx, w, g16, e, wl.lr)
+    elif variant == "momentum":
+        mom = torch.zeros(n, device=dev)
+        call = lambda: B.a2sgd_step_momentum(ctx, w, mom, g, e, wl.lr, 0.9, 1e-4)
+    elif variant == "replicated":
+        w_rep = B.padded_rows(P, n, dev)
+        w_rep.copy_(w.expand(P, n))
+        call = lambda: B.a2sgd_step(ctx, w_rep, g, e, wl.lr)
     elif variant == "segments":
         sizes = [sg.numel for sg in wl.segments]
         gs = [[t.clone() for t in torch.split(g[p], sizes)] for p in range(P)]
@@ -228,7 +254,7 @@ def run_variant(wl, variant, steps, warmup, dev):
         ws = [t.clone() for t in torch.split(w, sizes)]
         plan = B.a2sgd_segments_create(ctx, gs, es, ws)
         call = lambda: B.a2sgd_step_segments(ctx, plan, wl.lr)
-    else:  # deferred, single_launch: the step entry point of a context created with that flag
+    else:  # deferred, single_launch, misaligned: the step entry point on that context / layout
         call = lambda: B.a2sgd_step(ctx, w, g, e, wl.lr)
     for _ in range(max(3, warmup)):
         call()
@@ -674,7 +700,8 @@ def main():
     ap.add_argument("--scale-div", type=int, default=1,
                     help="divide every tensor length of the workload (small cases for profiler captures)")
     ap.add_argument("--variant", default="step",
-                    choices=["step", "dense_sync", "deferred", "bf16", "segments", "single_launch"],
+                    choices=["step", "dense_sync", "deferred", "bf16", "segments", "single_launch", "momentum",
+                             "replicated", "misaligned"],
                     help="with --minimal: which entry point the bare loop calls")
     ap.add_argument("--minimal", action="store_true",
                     help="timed step loop only (for profiler captures): no e2e, no per-kernel loop, "
@@ -810,7 +837,7 @@ def main():
     if exchange:
         line["exchange_between_gpus"] = exchange
     if not args.no_cpu_baseline and world == 1:
-        cb = oracle_sample_rate(wl, 10.0)
+        cb = oracle_sample_rate(wl, 10.0, all_cores=True)
         line["cpu_baseline"] = dict({k: v for k, v in cb.items() if not k.startswith("_")}, host=host_description())
     print(json.dumps(line), flush=True)
     if dist is not None:

@@ -72,6 +72,62 @@ def _load():
     return _lib
 
 
+_SRC_OMP = os.path.join(_HERE, "a2sgd_oracle_omp.c")
+_LIB_OMP = os.path.join(_HERE, "liba2sgd_oracle_omp.so")
+_lib_omp = None
+
+
+def build_omp(force: bool = False) -> str:
+    """Compile the OpenMP timing copy of the step (separate library; the pinned oracle is untouched)."""
+    if force or not os.path.exists(_LIB_OMP) or os.path.getmtime(_LIB_OMP) < os.path.getmtime(_SRC_OMP):
+        tmp = f"{_LIB_OMP}.{os.getpid()}.tmp"
+        subprocess.check_call(
+            ["gcc", "-O2", "-std=c11", "-fno-fast-math", "-ffp-contract=off", "-fopenmp",
+             "-shared", "-fPIC", "-o", tmp, _SRC_OMP])
+        os.replace(tmp, _LIB_OMP)
+    return _LIB_OMP
+
+
+def _load_omp():
+    global _lib_omp
+    if _lib_omp is None:
+        lib = ctypes.CDLL(build_omp())
+        f32p = ctypes.POINTER(ctypes.c_float)
+        lib.a2sgd_oracle_omp_threads.restype = ctypes.c_int
+        lib.a2sgd_oracle_omp_step.restype = ctypes.c_int
+        lib.a2sgd_oracle_omp_step.argtypes = [
+            ctypes.c_int, ctypes.c_uint64, ctypes.c_uint32, f32p, ctypes.c_int64,
+            f32p, ctypes.c_int64, f32p, ctypes.c_int64, ctypes.c_float,
+            f32p, f32p, ctypes.POINTER(ctypes.c_uint64)]
+        _lib_omp = lib
+    return _lib_omp
+
+
+def omp_threads() -> int:
+    """Threads the OpenMP copy will use."""
+    return int(_load_omp().a2sgd_oracle_omp_threads())
+
+
+def step_all_cores(w, grad, err, lr, *, mode=MODE_EF, n=None):
+    """The OpenMP timing copy of ``step`` (all host cores).  Same interface and, up to the order of
+    the fp64 additions inside the group sums, the same results."""
+    lib = _load_omp()
+    P = grad.shape[0]
+    n = grad.shape[1] if n is None else n
+    gp, gs = _rows(grad, "grad")
+    ep, es = _rows(err, "err") if err is not None else (None, 0)
+    wp, ws = _weights(w, P)
+    means = np.zeros((P, 2), np.float32)
+    gmeans = np.zeros(2, np.float32)
+    counts = np.zeros(P, np.uint64)
+    _check(lib.a2sgd_oracle_omp_step(
+        mode, n, P, wp, ws, gp, gs, ep, es, lr,
+        means.ctypes.data_as(ctypes.POINTER(ctypes.c_float)),
+        gmeans.ctypes.data_as(ctypes.POINTER(ctypes.c_float)),
+        counts.ctypes.data_as(ctypes.POINTER(ctypes.c_uint64))), "omp step")
+    return means, gmeans, counts
+
+
 def _rows(a: np.ndarray, name: str):
     """float32 [P, n] with unit inner stride -> (pointer, row stride in elements)."""
     if a.dtype != np.float32 or a.ndim != 2 or a.strides[1] != 4 or a.strides[0] % 4:

@@ -541,3 +541,25 @@ def test_momentum_bruteforce_rational(seed):
     # the shared state is the mean of the replica states (the update is linear)
     assert np.allclose(w, w_r.astype(np.float64).mean(0), rtol=0, atol=1e-6 * max(1.0, float(np.abs(w0).max())))
     assert np.allclose(m, m_r.astype(np.float64).mean(0), rtol=1e-6, atol=1e-6)
+
+
+# ---------------------------------------------------------------- the OpenMP timing copy of the step
+@pytest.mark.parametrize("mode", [EF, ALG1])
+@pytest.mark.parametrize("shared", [True, False])
+def test_all_cores_copy_agrees_with_the_pinned_oracle(mode, shared):
+    """bench.py times an OpenMP copy of the step next to the single-threaded oracle; the copy is
+    held to the pinned oracle here (it may differ only in the order of the fp64 additions)."""
+    rng = np.random.default_rng(17)
+    P, n = 3, 200_003
+    g = (rng.standard_normal((P, n)) * 1e-3).astype(np.float32)
+    g[rng.random((P, n)) < 0.05] = 0.0
+    e = (rng.standard_normal((P, n)) * 3e-4).astype(np.float32)
+    w = (rng.standard_normal(n if shared else (P, n)) * 0.02).astype(np.float32)
+    w1, e1 = w.copy(), e.copy()
+    lm1, gm1, c1 = oracle.step(w1, g, e1, 0.1, mode=mode)
+    w2, e2 = w.copy(), e.copy()
+    lm2, gm2, c2 = oracle.step_all_cores(w2, g, e2, 0.1, mode=mode)
+    assert np.array_equal(c1, c2)
+    assert np.allclose(lm1, lm2, rtol=2e-7, atol=0) and np.allclose(gm1, gm2, rtol=2e-7, atol=0)
+    assert np.allclose(w1, w2, rtol=0, atol=1e-9) and np.allclose(e1, e2, rtol=0, atol=1e-9)
+    assert oracle.omp_threads() >= 1
