@@ -45,10 +45,12 @@ UNIT = "params/s"
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 
-# DRAM bytes (read + write) per model element of the decode/update kernel, from the ncu
-# captures summarised under profiles/ (None until a capture exists for that P).
-NCU_DECODE_TRAFFIC_PER_ELEMENT = {4: 52.92}  # 36.0 read + 16.92 written inside the launch; 3.08 B/element of
-#                                               dirty lines leave L2 during the next launch
+# DRAM bytes (read + write) per model element of the decode/update kernel inside one launch, from the
+# ncu captures summarised under profiles/ (step_kernels_c2_lstm_ptb_div4.md for P = 4,
+# step_kernels_c3_resnet50_div4.md for P = 8): reads equal the algorithmic (8P + 4) bytes; of the
+# (4P + 4) bytes written about 3 (P = 4) to 7.5 (P = 8) bytes per element are still dirty in L2 when
+# the kernel ends and leave during the next launch.
+NCU_DECODE_TRAFFIC_PER_ELEMENT = {4: 36.00 + 16.78, 8: 68.00 + 28.49}
 DEFAULT_WORKLOAD = "c5_gpt2_xl"
 FALLBACK_WORKLOAD = "c4_vgg16"
 
