@@ -450,6 +450,7 @@ def time_workload(wl, steps, warmup, dev, *, with_roofline=True, with_next_rows=
             ws = [t.clone() for t in torch.split(w, sizes)]
             plan = B.a2sgd_segments_create(ctx, gs, es, ws)
             res["step_segments_ms"] = timed(lambda: B.a2sgd_step_segments(ctx, plan, wl.lr))
+            res["step_segments_per_tensor_ms"] = timed(lambda: B.a2sgd_step_segments_per_tensor(ctx, plan, wl.lr))
             plan.destroy()
             del gs, es, ws, plan
             torch.cuda.empty_cache()
@@ -554,6 +555,12 @@ def next_rows_of(wl, res, peak_gbs) -> dict:
         rows["step over a segment list (one tensor per segment)"] = {
             "ms": res["step_segments_ms"], "GBps": bts / (res["step_segments_ms"] * 1e-3) / 1e9,
             "frac_of_8TBps": bts / (res["step_segments_ms"] * 1e-3) / 1e9 / NOMINAL_HBM_GBS,
+            "segments": len(wl.segments)}
+    if "step_segments_per_tensor_ms" in res:
+        bts = b["step"] * wl.n
+        rows["step over a segment list, every tensor compressed on its own (2S floats per worker)"] = {
+            "ms": res["step_segments_per_tensor_ms"], "GBps": bts / (res["step_segments_per_tensor_ms"] * 1e-3) / 1e9,
+            "frac_of_8TBps": bts / (res["step_segments_per_tensor_ms"] * 1e-3) / 1e9 / NOMINAL_HBM_GBS,
             "segments": len(wl.segments)}
     if "step_deferred_ms" in res:
         bts = (12 * wl.P + 8 + wl.P / 4) * wl.n

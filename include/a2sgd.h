@@ -282,6 +282,22 @@ int a2sgd_step_segments(a2sgd_ctx *ctx, a2sgd_segments *plan, float lr, void *st
  * paper's experimental setup for VGG-16); computing those rates is the caller's business. */
 int a2sgd_step_segments_lr(a2sgd_ctx *ctx, a2sgd_segments *plan, const float *lr_per_segment, void *stream);
 
+/* The per-tensor variant of a2sgd_step_segments: every tensor of the list is compressed on its own,
+ * as if Algorithm 1 (lines 3-7) were run once per tensor — tensor s has its own pair of local means
+ * per worker, its own pair of global means (the unweighted average over the workers), and is
+ * reconstructed from those.  The payload a worker would exchange grows from 2 to 2S floats: this is
+ * NOT the method's whole-model reading (Section 4.3 takes the two averages over all gradients of the
+ * model) but the granularity a per-tensor communication layer works at; results equal a2sgd_step
+ * called separately on every tensor.  Three launches (encode per tile, fold per tensor,
+ * decode/update).  The first call on a plan allocates the variant's scratch (24 bytes per worker
+ * and 2048-element tile, plus the per-tensor means).  lr_per_segment: DEVICE [S] or NULL.
+ * a2sgd_read_segment_stats synchronises `stream` and copies the per-tensor results to HOST memory:
+ *   local_means_host [S][P][2], global_means_host [S][2], pos_counts_host [S][P]; any may be NULL. */
+int a2sgd_step_segments_per_tensor(a2sgd_ctx *ctx, a2sgd_segments *plan, float lr, const float *lr_per_segment,
+                                   void *stream);
+int a2sgd_read_segment_stats(a2sgd_ctx *ctx, a2sgd_segments *plan, float *local_means_host,
+                             float *global_means_host, uint64_t *pos_counts_host, void *stream);
+
 /* The two stages of a2sgd_step_segments as separate calls, mirroring a2sgd_encode and
  * a2sgd_decode_update (Algorithm 1 line 3, and lines 4, 6, 7) for a segment list; the 2P scalars
  * are averaged in between with a2sgd_global_average (line 5).

@@ -96,6 +96,10 @@ def lib() -> ctypes.CDLL:
         l.a2sgd_encode_segments.argtypes = [_vp, _vp, _vp, _vp, _vp]
         l.a2sgd_decode_update_segments.restype = ctypes.c_int
         l.a2sgd_decode_update_segments.argtypes = [_vp, _vp, _vp, _vp, ctypes.c_float, _vp, _vp]
+        l.a2sgd_step_segments_per_tensor.restype = ctypes.c_int
+        l.a2sgd_step_segments_per_tensor.argtypes = [_vp, _vp, ctypes.c_float, _vp, _vp]
+        l.a2sgd_read_segment_stats.restype = ctypes.c_int
+        l.a2sgd_read_segment_stats.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp]
         l.a2sgd_step_segments.restype = ctypes.c_int
         l.a2sgd_step_segments.argtypes = [_vp, _vp, ctypes.c_float, _vp]
         for fn in (l.a2sgd_step_bf16, l.a2sgd_step_f16):
@@ -396,6 +400,25 @@ def a2sgd_decode_update_segments(ctx: Context, plan: Segments, local_means: Opti
                                               global_means.data_ptr(), float(lr),
                                               lr_per_segment.data_ptr() if lr_per_segment is not None else None,
                                               _stream(stream)), "a2sgd_decode_update_segments")
+
+
+def a2sgd_step_segments_per_tensor(ctx: Context, plan: Segments, lr: float,
+                                   lr_per_segment: Optional[torch.Tensor] = None, stream=None) -> None:
+    """Every tensor compressed on its own (its own local and global means)."""
+    _check(lib().a2sgd_step_segments_per_tensor(ctx.handle, plan.handle, float(lr),
+                                                lr_per_segment.data_ptr() if lr_per_segment is not None else None,
+                                                _stream(stream)), "a2sgd_step_segments_per_tensor")
+
+
+def a2sgd_read_segment_stats(ctx: Context, plan: Segments, S: int, stream=None):
+    """Synchronises the stream.  Returns (local_means [S,P,2], global_means [S,2], pos_counts [S,P])."""
+    import numpy as np
+    lm = np.zeros((S, ctx.P, 2), np.float32)
+    gm = np.zeros((S, 2), np.float32)
+    pc = np.zeros((S, ctx.P), np.uint64)
+    _check(lib().a2sgd_read_segment_stats(ctx.handle, plan.handle, lm.ctypes.data, gm.ctypes.data, pc.ctypes.data,
+                                          _stream(stream)), "a2sgd_read_segment_stats")
+    return lm, gm, pc
 
 
 def a2sgd_step_segments_lr(ctx: Context, plan: Segments, lr_per_segment: torch.Tensor, stream=None) -> None:

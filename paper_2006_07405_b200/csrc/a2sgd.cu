@@ -73,8 +73,13 @@ struct a2sgd_segments {
     bool has_err = false;
     // device tables
     SegTile *tiles = nullptr;
-    SegStart *starts = nullptr; // [S + 1], only for S <= kSegScanMax
+    SegStart *starts = nullptr; // [S + 1]
     uint64_t n_tiles = 0;
+    // scratch of the per-tensor-means variant, allocated by its first call
+    Partial *tile_partials = nullptr;          // [P][n_tiles]
+    float *seg_local_means = nullptr;          // [S][P][2]
+    unsigned long long *seg_counts = nullptr;  // [S][P]
+    float *seg_global_means = nullptr;         // [S][2]
     uint64_t *numel = nullptr;
     const float **grad = nullptr;
     float **err = nullptr;
@@ -919,11 +924,9 @@ extern "C" int a2sgd_segments_create(a2sgd_ctx *c, uint32_t S, const uint64_t *n
     ok = ok && cudaMalloc(&sg->w, sizeof(float *) * w_count) == cudaSuccess;
     if (err) ok = ok && cudaMalloc(&sg->err, sizeof(float *) * (size_t)P * S) == cudaSuccess;
     ok = ok && cudaMemcpy(sg->tiles, tiles.data(), sizeof(SegTile) * tiles.size(), cudaMemcpyHostToDevice) == cudaSuccess;
-    if (S <= kSegScanMax) {
-        starts.push_back(SegStart{(uint64_t)tiles.size(), 0, 0u, {0u, 0u, 0u}}); // end marker
-        ok = ok && cudaMalloc(&sg->starts, sizeof(SegStart) * starts.size()) == cudaSuccess;
-        ok = ok && cudaMemcpy(sg->starts, starts.data(), sizeof(SegStart) * starts.size(), cudaMemcpyHostToDevice) == cudaSuccess;
-    }
+    starts.push_back(SegStart{(uint64_t)tiles.size(), 0, 0u, {0u, 0u, 0u}}); // end marker
+    ok = ok && cudaMalloc(&sg->starts, sizeof(SegStart) * starts.size()) == cudaSuccess;
+    ok = ok && cudaMemcpy(sg->starts, starts.data(), sizeof(SegStart) * starts.size(), cudaMemcpyHostToDevice) == cudaSuccess;
     ok = ok && cudaMemcpy(sg->numel, numel, sizeof(uint64_t) * S, cudaMemcpyHostToDevice) == cudaSuccess;
     ok = ok && cudaMemcpy(sg->grad, grad, sizeof(float *) * (size_t)P * S, cudaMemcpyHostToDevice) == cudaSuccess;
     ok = ok && cudaMemcpy(sg->w, w, sizeof(float *) * w_count, cudaMemcpyHostToDevice) == cudaSuccess;
@@ -943,6 +946,10 @@ extern "C" int a2sgd_segments_destroy(a2sgd_segments *sg)
     DeviceGuard guard(sg->ctx->device);
     cudaFree(sg->tiles);
     cudaFree(sg->starts);
+    cudaFree(sg->tile_partials);
+    cudaFree(sg->seg_local_means);
+    cudaFree(sg->seg_counts);
+    cudaFree(sg->seg_global_means);
     cudaFree(sg->numel);
     cudaFree(sg->grad);
     cudaFree(sg->err);
@@ -956,7 +963,12 @@ static SegTables seg_tables(const a2sgd_segments *sg, const float *lr_per_segmen
 {
     SegTables t{};
     t.tiles = sg->tiles;
-    t.starts = sg->starts;
+    t.starts = sg->S <= kSegScanMax ? sg->starts : nullptr; // beyond that the decode kernel reads the tile table
+    t.all_starts = sg->starts;
+    t.tile_partials = sg->tile_partials;
+    t.seg_local_means = sg->seg_local_means;
+    t.seg_counts = sg->seg_counts;
+    t.seg_global_means = sg->seg_global_means;
     t.n_tiles = sg->n_tiles;
     t.numel = sg->numel;
     t.grad = sg->grad;
@@ -969,11 +981,12 @@ static SegTables seg_tables(const a2sgd_segments *sg, const float *lr_per_segmen
 }
 
 static int launch_encode_segments(a2sgd_ctx *c, a2sgd_segments *sg, float *local_means,
-                                  unsigned long long *pos_counts, float *global_means, cudaStream_t s)
+                                  unsigned long long *pos_counts, float *global_means, cudaStream_t s,
+                                  bool per_tensor = false)
 {
     SegTables t = seg_tables(sg, nullptr);
     EncodeArgs a = make_encode_args(c, nullptr, 0, nullptr, 0, local_means, pos_counts, nullptr, global_means);
-    const void *fn = c->k->encode_segments(!c->alg1);
+    const void *fn = c->k->encode_segments(!c->alg1, per_tensor);
     const uint64_t slots = (uint64_t)c->sm_count * occupancy(c, fn) * kWavesK1;
     uint64_t G = std::max<uint64_t>(1, slots / c->P);
     G = std::min<uint64_t>(std::min<uint64_t>(G, sg->n_tiles), c->g_alloc);
@@ -983,14 +996,15 @@ static int launch_encode_segments(a2sgd_ctx *c, a2sgd_segments *sg, float *local
 }
 
 static int launch_decode_segments(a2sgd_ctx *c, a2sgd_segments *sg, const float *local_means,
-                                  const float *global_means, float lr, const float *lr_per_segment, cudaStream_t s)
+                                  const float *global_means, float lr, const float *lr_per_segment, cudaStream_t s,
+                                  bool per_tensor = false)
 {
     const bool ef = !c->alg1;
     const bool store = ef || sg->has_err;
     SegTables t = seg_tables(sg, lr_per_segment);
     DecodeArgs a = make_decode_args(c, nullptr, sg->replicated ? 1 : 0, nullptr, 0, nullptr, 0, local_means,
                                     global_means, lr);
-    const void *fn = c->k->decode_segments(ef, store, c->P);
+    const void *fn = c->k->decode_segments(ef, store, c->P, per_tensor);
     const uint64_t grid = std::min<uint64_t>(sg->n_tiles, 0x7fffffffu);
     void *params[] = {&a, &t};
     A2_CUDA(launch_pdl(fn, dim3((unsigned)grid), params, s));
@@ -1020,6 +1034,75 @@ extern "C" int a2sgd_step_segments_lr(a2sgd_ctx *c, a2sgd_segments *sg, const fl
 {
     if (!lr_per_segment || !aligned(lr_per_segment, 4)) return lr_per_segment ? A2SGD_ERR_ALIGN : A2SGD_ERR_ARG;
     return step_segments_impl(c, sg, 0.0f, lr_per_segment, stream);
+}
+
+// Scratch of the per-tensor-means variant: one partial per (worker, tile), the per-tensor means and counts.
+static int ensure_per_tensor_scratch(a2sgd_ctx *c, a2sgd_segments *sg)
+{
+    if (sg->tile_partials) return A2SGD_OK;
+    const size_t P = c->P, S = sg->S;
+    bool ok = true;
+    ok = ok && cudaMalloc(&sg->tile_partials, sizeof(Partial) * P * sg->n_tiles) == cudaSuccess;
+    ok = ok && cudaMalloc(&sg->seg_local_means, sizeof(float) * 2 * P * S) == cudaSuccess;
+    ok = ok && cudaMalloc(&sg->seg_counts, sizeof(unsigned long long) * P * S) == cudaSuccess;
+    ok = ok && cudaMalloc(&sg->seg_global_means, sizeof(float) * 2 * S) == cudaSuccess;
+    if (!ok) {
+        (void)cudaGetLastError();
+        cudaFree(sg->tile_partials);
+        cudaFree(sg->seg_local_means);
+        cudaFree(sg->seg_counts);
+        cudaFree(sg->seg_global_means);
+        sg->tile_partials = nullptr;
+        sg->seg_local_means = sg->seg_global_means = nullptr;
+        sg->seg_counts = nullptr;
+        (void)cudaGetLastError();
+        return A2SGD_ERR_NOMEM;
+    }
+    return A2SGD_OK;
+}
+
+extern "C" int a2sgd_step_segments_per_tensor(a2sgd_ctx *c, a2sgd_segments *sg, float lr, const float *lr_per_segment,
+                                              void *stream)
+{
+    if (!c || !sg || sg->ctx != c) return A2SGD_ERR_ARG;
+    if (lr_per_segment && !aligned(lr_per_segment, 4)) return A2SGD_ERR_ALIGN;
+    if (lr_per_segment && !device_pointer_ok(c, lr_per_segment)) return A2SGD_ERR_ARG;
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return A2SGD_ERR_CUDA;
+    const int rc0 = ensure_per_tensor_scratch(c, sg);
+    if (rc0) return rc0;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    DebugScope dbg(c, s);
+    if (!dbg.arm(2)) return A2SGD_ERR_CUDA;
+    const int rc = launch_encode_segments(c, sg, c->local_means, c->pos_counts, nullptr, s, true);
+    if (rc) return rc;
+    {
+        SegTables t = seg_tables(sg, nullptr);
+        uint32_t P = c->P;
+        int *status = c->status;
+        void *params[] = {&t, &P, &status};
+        A2_CUDA(launch_pdl(c->k->fold_segments, dim3(sg->S), params, s));
+    }
+    return launch_decode_segments(c, sg, nullptr, nullptr, lr, lr_per_segment, s, true);
+}
+
+extern "C" int a2sgd_read_segment_stats(a2sgd_ctx *c, a2sgd_segments *sg, float *local_means_host,
+                                        float *global_means_host, uint64_t *pos_counts_host, void *stream)
+{
+    if (!c || !sg || sg->ctx != c) return A2SGD_ERR_ARG;
+    if (!sg->tile_partials) return A2SGD_ERR_ARG; // no per-tensor step has run on this plan
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return A2SGD_ERR_CUDA;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const size_t P = c->P, S = sg->S;
+    if (local_means_host)
+        A2_CUDA(cudaMemcpyAsync(local_means_host, sg->seg_local_means, sizeof(float) * 2 * P * S, cudaMemcpyDeviceToHost, s));
+    if (global_means_host)
+        A2_CUDA(cudaMemcpyAsync(global_means_host, sg->seg_global_means, sizeof(float) * 2 * S, cudaMemcpyDeviceToHost, s));
+    if (pos_counts_host)
+        A2_CUDA(cudaMemcpyAsync(pos_counts_host, sg->seg_counts, sizeof(uint64_t) * P * S, cudaMemcpyDeviceToHost, s));
+    A2_CUDA(cudaStreamSynchronize(s));
+    return A2SGD_OK;
 }
 
 extern "C" int a2sgd_encode_segments(a2sgd_ctx *c, a2sgd_segments *sg, float *local_means, uint64_t *pos_counts,

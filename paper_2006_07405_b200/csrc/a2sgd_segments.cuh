@@ -47,6 +47,12 @@ struct SegTables {
     uint32_t S;
     uint32_t w_replicated;
     const float *lr_per_segment; // [S] device, or nullptr: one learning rate for the whole model
+    // per-tensor-means variant only (plan-owned scratch)
+    const SegStart *all_starts;        // [S + 1], always present
+    Partial *tile_partials;            // [P][n_tiles]
+    float *seg_local_means;            // [S][P][2]
+    unsigned long long *seg_counts;    // [S][P]
+    float *seg_global_means;           // [S][2]
 };
 
 // An entry of a pointer table through the read-only (L1-cached) path: the tables are small and every
@@ -58,7 +64,10 @@ __device__ __forceinline__ T *ld_ptr(T *const *slot)
 }
 
 // K1 over a segment list.  grid = (G, P); CTA x walks tiles x, x + G, ...
-template <bool EF>
+// PER_TENSOR: every tensor keeps its own pair of means, so the sums are not carried across tiles:
+// each tile's (S+, S-, n+) goes to its own slot of t.tile_partials and k_fold_segments adds the
+// slots of a tensor in tile order afterwards.
+template <bool EF, bool PER_TENSOR = false>
 __global__ void __launch_bounds__(kBlock) k_encode_segments(EncodeArgs a, SegTables t)
 {
     pdl_wait_prior_grid();
@@ -69,6 +78,7 @@ __global__ void __launch_bounds__(kBlock) k_encode_segments(EncodeArgs a, SegTab
     const uint32_t p = blockIdx.y;
     Acc acc;
     for (uint64_t tile = blockIdx.x; tile < t.n_tiles; tile += gridDim.x) {
+        if (PER_TENSOR) acc = Acc();
         const SegTile d = t.tiles[tile];
         if (d.seg >= t.S) {                     // only reachable with a corrupt table
             span_ok(d.seg, 1, t.S);
@@ -118,24 +128,83 @@ __global__ void __launch_bounds__(kBlock) k_encode_segments(EncodeArgs a, SegTab
         }
         acc.s_pos += (double)sp;
         acc.s_neg += (double)sn;
+        if (PER_TENSOR) {
+            double s_pos = acc.s_pos, s_neg = acc.s_neg;
+            unsigned long long n_pos = acc.n_pos;
+            block_reduce(s_pos, s_neg, n_pos, sh_d, sh_n);
+            if (threadIdx.x == 0) {
+                Partial &slot = t.tile_partials[(uint64_t)p * t.n_tiles + tile];
+                slot.s_pos = s_pos;
+                slot.s_neg = s_neg;
+                slot.n_pos = n_pos;
+            }
+        }
     }
+    if (PER_TENSOR) return;
     double s_pos = acc.s_pos, s_neg = acc.s_neg;
     unsigned long long n_pos = acc.n_pos;
     block_reduce(s_pos, s_neg, n_pos, sh_d, sh_n);
     finish_worker(a, p, s_pos, s_neg, n_pos, sh_d, sh_n, &sh_flag);
 }
 
-// K3 over a segment list: one tile per CTA.  PT > 0: compile-time worker count.
-template <bool EF, bool STORE, int PT>
+// Per-tensor-means variant, between K1 and K3: block s adds the tile slots of tensor s in tile
+// order (thread t takes slots t, t + 256, ...; fixed tree above), one worker after the other, writes
+// that tensor's local means and counts, and averages them over the workers in worker order
+// (Algorithm 1 line 5, once per tensor).  grid = S.
+static __global__ void __launch_bounds__(kBlock) k_fold_segments(SegTables t, uint32_t P, int *status)
+{
+    pdl_wait_prior_grid();
+    pdl_release_next_grid();
+    __shared__ double sh_d[2][kWarps];
+    __shared__ unsigned long long sh_n[kWarps];
+    const uint32_t sg = blockIdx.x;
+    const uint64_t first = t.all_starts[sg].first_tile, last = t.all_starts[sg + 1].first_tile;
+    const uint64_t numel = t.all_starts[sg].numel;
+    double g_pos = 0.0, g_neg = 0.0; // thread 0: sums of the workers' means
+    for (uint32_t p = 0; p < P; ++p) {
+        const Partial *slot = t.tile_partials + (uint64_t)p * t.n_tiles;
+        double s_pos = 0.0, s_neg = 0.0;
+        unsigned long long n_pos = 0;
+        for (uint64_t i = first + threadIdx.x; i < last; i += kBlock) {
+            s_pos += __ldcg(&slot[i].s_pos);
+            s_neg += __ldcg(&slot[i].s_neg);
+            n_pos += __ldcg(&slot[i].n_pos);
+        }
+        block_reduce(s_pos, s_neg, n_pos, sh_d, sh_n);
+        if (threadIdx.x == 0) {
+            const unsigned long long n_neg = numel - n_pos;
+            const float mu_pos = n_pos ? (float)(s_pos / (double)n_pos) : 0.0f;
+            const float mu_neg = n_neg ? (float)(s_neg / (double)n_neg) : 0.0f;
+            if (!isfinite(s_pos) || !isfinite(s_neg)) atomicCAS(status, kDevOk, kDevNonFinite);
+            t.seg_local_means[((uint64_t)sg * P + p) * 2 + 0] = mu_pos;
+            t.seg_local_means[((uint64_t)sg * P + p) * 2 + 1] = mu_neg;
+            t.seg_counts[(uint64_t)sg * P + p] = n_pos;
+            g_pos += (double)mu_pos;
+            g_neg += (double)mu_neg;
+        }
+    }
+    if (threadIdx.x == 0) {
+        t.seg_global_means[2 * sg + 0] = (float)(g_pos / (double)P);
+        t.seg_global_means[2 * sg + 1] = (float)(g_neg / (double)P);
+    }
+}
+
+// K3 over a segment list: one tile per CTA.  PT > 0: compile-time worker count.  PER_TENSOR: the
+// means of the tile's own tensor (written by k_fold_segments) instead of the whole-model means.
+template <bool EF, bool STORE, int PT, bool PER_TENSOR = false>
 __global__ void __launch_bounds__(kBlock) k_decode_segments(DecodeArgs a, SegTables t)
 {
     pdl_wait_prior_grid();
     pdl_release_next_grid();
     __shared__ WorkerConst sh_c[PT > 0 ? 1 : kMaxP];
     const uint32_t P = PT > 0 ? PT : a.P;
-    const float m_pos = __ldg(a.global_means), m_neg = __ldg(a.global_means + 1);
+    float m_pos = 0.f, m_neg = 0.f;
+    if (!PER_TENSOR) {
+        m_pos = __ldg(a.global_means);
+        m_neg = __ldg(a.global_means + 1);
+    }
     const bool repl = t.w_replicated != 0;
-    if (PT == 0) {
+    if (PT == 0 && !PER_TENSOR) {
         for (uint32_t p = threadIdx.x; p < P; p += kBlock) sh_c[p] = worker_const<EF>(a, p, m_pos, m_neg);
         __syncthreads();
     }
@@ -161,6 +230,16 @@ __global__ void __launch_bounds__(kBlock) k_decode_segments(DecodeArgs a, SegTab
             n_s = __ldg(t.numel + d.seg);
         }
         if (!span_ok(d.offset, 1, n_s)) continue; // the tile starts inside its tensor
+        if (PER_TENSOR) {
+            m_pos = __ldcg(t.seg_global_means + 2 * d.seg);
+            m_neg = __ldcg(t.seg_global_means + 2 * d.seg + 1);
+            a.local_means = t.seg_local_means + (uint64_t)d.seg * P * 2; // this tensor's P pairs
+            if (PT == 0) {
+                __syncthreads();
+                for (uint32_t p = threadIdx.x; p < P; p += kBlock) sh_c[p] = worker_const<EF>(a, p, m_pos, m_neg);
+                __syncthreads();
+            }
+        }
         const uint64_t i = d.offset + (uint64_t)threadIdx.x * kSegVW;
         // layer-wise learning rates (e.g. LARS, which the paper uses for VGG-16): one per tensor
         const float lr = t.lr_per_segment ? __ldg(t.lr_per_segment + d.seg) : a.lr;

@@ -174,18 +174,17 @@ const void *select_decode_deferred(uint32_t P)
     }
 }
 
-template <bool EF, bool STORE>
+template <bool EF, bool STORE, bool PER_TENSOR>
 const void *select_decode_segments_p(uint32_t P)
 {
     switch (P) {
-    case 1: return (const void *)k_decode_segments<EF, STORE, 1>;
-    case 2: return (const void *)k_decode_segments<EF, STORE, 2>;
-    case 4: return (const void *)k_decode_segments<EF, STORE, 4>;
-    case 8: return (const void *)k_decode_segments<EF, STORE, 8>;
-    default: return (const void *)k_decode_segments<EF, STORE, 0>;
+    case 1: return (const void *)k_decode_segments<EF, STORE, 1, PER_TENSOR>;
+    case 2: return (const void *)k_decode_segments<EF, STORE, 2, PER_TENSOR>;
+    case 4: return (const void *)k_decode_segments<EF, STORE, 4, PER_TENSOR>;
+    case 8: return (const void *)k_decode_segments<EF, STORE, 8, PER_TENSOR>;
+    default: return (const void *)k_decode_segments<EF, STORE, 0, PER_TENSOR>;
     }
 }
-
 
 inline const void *table_encode_deferred(bool holds_v)
 {
@@ -195,9 +194,10 @@ inline const void *table_encode_lowp(int gt, bool ef, int vw)
 {
     return gt == 1 ? select_encode_lowp<1>(ef, vw) : select_encode_lowp<2>(ef, vw);
 }
-inline const void *table_encode_segments(bool ef)
+inline const void *table_encode_segments(bool ef, bool per_tensor)
 {
-    return ef ? (const void *)k_encode_segments<true> : (const void *)k_encode_segments<false>;
+    if (per_tensor) return ef ? (const void *)k_encode_segments<true, true> : (const void *)k_encode_segments<false, true>;
+    return ef ? (const void *)k_encode_segments<true, false> : (const void *)k_encode_segments<false, false>;
 }
 inline const void *table_decode_lowp(int gt, bool ef, bool store, bool shared, uint32_t P, int vw)
 {
@@ -207,10 +207,16 @@ inline const void *table_decode_deferred(bool repl, uint32_t P)
 {
     return repl ? select_decode_deferred<true>(P) : select_decode_deferred<false>(P);
 }
-inline const void *table_decode_segments(bool ef, bool store, uint32_t P)
+template <bool PER_TENSOR>
+const void *table_decode_segments_m(bool ef, bool store, uint32_t P)
 {
-    return ef ? select_decode_segments_p<true, true>(P)
-              : store ? select_decode_segments_p<false, true>(P) : select_decode_segments_p<false, false>(P);
+    return ef ? select_decode_segments_p<true, true, PER_TENSOR>(P)
+              : store ? select_decode_segments_p<false, true, PER_TENSOR>(P)
+                      : select_decode_segments_p<false, false, PER_TENSOR>(P);
+}
+inline const void *table_decode_segments(bool ef, bool store, uint32_t P, bool per_tensor)
+{
+    return per_tensor ? table_decode_segments_m<true>(ef, store, P) : table_decode_segments_m<false>(ef, store, P);
 }
 
 inline a2sgd_kernel_table kernel_table()
@@ -232,6 +238,7 @@ inline a2sgd_kernel_table kernel_table()
     t.global_average = (const void *)k_global_average;
     t.global_average_from_sums = (const void *)k_global_average_from_sums;
     t.materialize_err = (const void *)k_materialize_err;
+    t.fold_segments = (const void *)k_fold_segments;
     return t;
 }
 

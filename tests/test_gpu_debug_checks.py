@@ -85,6 +85,7 @@ def test_checked_segment_list_kernels():
         ctx = B.a2sgd_create(n, P, 0, EF | dbg)
         plan = B.a2sgd_segments_create(ctx, grad, err, w)
         B.a2sgd_step_segments(ctx, plan, 0.1)
+        B.a2sgd_step_segments_per_tensor(ctx, plan, 0.1)
         *_, status = B.a2sgd_read_stats(ctx)
         assert status == B.OK
         outs.append(torch.cat(w + [t for row in err for t in row]).cpu().numpy().tobytes())

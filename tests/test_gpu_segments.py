@@ -230,3 +230,78 @@ def test_alg1_error_table_with_a_missing_entry_is_rejected():
     rc = B.lib().a2sgd_segments_create(ctx.handle, 2, numel, g_tab, e_tab, w_tab, 0, ctypes.byref(out))
     assert rc == B.ERR_ARG and not out
     ctx.destroy()
+
+
+@pytest.mark.parametrize("mode", [EF, ALG1])
+@pytest.mark.parametrize("replicated", [False, True])
+@pytest.mark.parametrize("P,offsets", [(1, [0]), (4, [0]), (3, [0, 1, 0, 8, 3]), (8, [0, 0, 2])])
+def test_per_tensor_means_variant_equals_one_oracle_step_per_tensor(mode, replicated, P, offsets):
+    """a2sgd_step_segments_per_tensor compresses every tensor on its own: the reference is the
+    oracle's step called once per tensor (its own local means, its own global means)."""
+    sizes = [1, 5, 2047, 2048, 2049, 70_001, 33, 3 * 2048, 12_345, 64]
+    S = len(sizes)
+    gen = torch.Generator("cuda").manual_seed(31 * P + len(offsets))
+    grad = [_tensors(sizes, offsets, gen, 1e-3) for _ in range(P)]
+    for p in range(P):                      # a different scale per tensor, so per-tensor means really differ
+        for k, t in enumerate(grad[p]):
+            t.mul_(10.0 ** (k % 4))
+    err = [_tensors(sizes, offsets, gen, 3e-4) for _ in range(P)]
+    w = [_tensors(sizes, offsets, gen, 0.02) for _ in range(P if replicated else 1)]
+    lrs = torch.tensor([0.1 * (1 + k % 3) for k in range(S)], device="cuda")
+    # reference: one oracle step per tensor
+    refs = []
+    for k in range(S):
+        g_k = np.stack([grad[p][k].cpu().numpy() for p in range(P)])
+        e_k = np.stack([err[p][k].cpu().numpy() for p in range(P)])
+        w_k = np.stack([w[p][k].cpu().numpy() for p in range(P)]) if replicated else w[0][k].cpu().numpy().copy()
+        lm, gm, cnt = oracle.step(w_k, g_k, e_k, float(lrs[k]), mode=mode)
+        refs.append((lm, gm, cnt, w_k, e_k))
+    ctx = B.a2sgd_create(sum(sizes), P, 0, mode)
+    plan = B.a2sgd_segments_create(ctx, grad, err, w if replicated else w[0], w_replicated=replicated)
+    B.a2sgd_step_segments_per_tensor(ctx, plan, 0.0, lrs)
+    lm_all, gm_all, cnt_all = B.a2sgd_read_segment_stats(ctx, plan, S)
+    *_, status = B.a2sgd_read_stats(ctx)
+    assert status == B.OK
+    for k, (lm, gm, cnt, w_k, e_k) in enumerate(refs):
+        assert np.array_equal(cnt_all[k], cnt), f"tensor {k} counts"
+        assert_means(lm_all[k], lm, f"tensor {k} local means")
+        assert_means(gm_all[k], gm, f"tensor {k} global means")
+        w_got = np.stack([w[p][k].cpu().numpy() for p in range(P)]) if replicated else w[0][k].cpu().numpy()
+        e_got = np.stack([err[p][k].cpu().numpy() for p in range(P)])
+        assert_state(w_got, w_k, e_got, e_k, gm, f"tensor {k}")
+    for rows in (grad, err, w):                              # nothing written outside the tensors
+        for row in rows:
+            for t in row:
+                full = torch.tensor([], dtype=torch.float32, device="cuda").set_(t.untyped_storage())
+                o = t.storage_offset()
+                assert torch.isnan(full[:o]).all() and torch.isnan(full[o + t.numel():]).all()
+    # a second step on the same plan reuses the scratch and stays reproducible
+    B.a2sgd_step_segments_per_tensor(ctx, plan, 0.0, lrs)
+    *_, status = B.a2sgd_read_stats(ctx)
+    assert status == B.OK
+    plan.destroy()
+    ctx.destroy()
+
+
+def test_per_tensor_variant_with_equal_tensors_matches_whole_model_step():
+    """If every tensor holds the same values, per-tensor means equal whole-model means, so the two
+    variants must produce the same weights (to rounding of the differently ordered sums)."""
+    P, n_t, S = 2, 4096, 3
+    gen = torch.Generator("cuda").manual_seed(8)
+    g0 = [torch.empty(n_t, device="cuda").normal_(0, 1e-3, generator=gen) for _ in range(P)]
+    outs = []
+    for variant in ("whole", "per_tensor"):
+        grad = [[g0[p].clone() for _ in range(S)] for p in range(P)]
+        err = [[torch.zeros(n_t, device="cuda") for _ in range(S)] for _ in range(P)]
+        w = [torch.ones(n_t, device="cuda") for _ in range(S)]
+        ctx = B.a2sgd_create(n_t * S, P, 0, EF)
+        plan = B.a2sgd_segments_create(ctx, grad, err, w)
+        if variant == "whole":
+            B.a2sgd_step_segments(ctx, plan, 0.1)
+        else:
+            B.a2sgd_step_segments_per_tensor(ctx, plan, 0.1)
+        torch.cuda.synchronize()
+        outs.append(torch.cat(w).cpu().numpy())
+        plan.destroy()
+        ctx.destroy()
+    assert np.allclose(outs[0], outs[1], rtol=0, atol=1e-9)
