@@ -288,7 +288,7 @@ int a2sgd_step_segments_lr(a2sgd_ctx *ctx, a2sgd_segments *plan, const float *lr
  * reconstructed from those.  The payload a worker would exchange grows from 2 to 2S floats: this is
  * NOT the method's whole-model reading (Section 4.3 takes the two averages over all gradients of the
  * model) but the granularity a per-tensor communication layer works at; results equal a2sgd_step
- * called separately on every tensor.  Three launches (encode per tile, fold per tensor,
+ * called separately on every tensor.  Four launches (encode per tile, two-level fold per tensor,
  * decode/update).  The first call on a plan allocates the variant's scratch (24 bytes per worker
  * and 2048-element tile, plus the per-tensor means).  lr_per_segment: DEVICE [S] or NULL.
  * a2sgd_read_segment_stats synchronises `stream` and copies the per-tensor results to HOST memory:

@@ -76,7 +76,10 @@ struct a2sgd_segments {
     SegStart *starts = nullptr; // [S + 1]
     uint64_t n_tiles = 0;
     // scratch of the per-tensor-means variant, allocated by its first call
+    FoldJob *fold_jobs = nullptr;              // [n_jobs], built with the plan
+    uint32_t n_jobs = 0;
     Partial *tile_partials = nullptr;          // [P][n_tiles]
+    Partial *job_partials = nullptr;           // [P][n_jobs]
     float *seg_local_means = nullptr;          // [S][P][2]
     unsigned long long *seg_counts = nullptr;  // [S][P]
     float *seg_global_means = nullptr;         // [S][2]
@@ -884,6 +887,7 @@ extern "C" int a2sgd_segments_create(a2sgd_ctx *c, uint32_t S, const uint64_t *n
     uint64_t total = 0;
     std::vector<SegTile> tiles;
     std::vector<SegStart> starts;
+    std::vector<FoldJob> jobs;
     for (uint32_t s = 0; s < S; ++s) {
         if (numel[s] == 0) return A2SGD_ERR_ARG;
         total += numel[s];
@@ -903,8 +907,11 @@ extern "C" int a2sgd_segments_create(a2sgd_ctx *c, uint32_t S, const uint64_t *n
             if (!aligned(wp, 4)) return A2SGD_ERR_ALIGN;
             vec = vec && aligned(wp, 32);
         }
-        starts.push_back(SegStart{(uint64_t)tiles.size(), numel[s], vec ? kSegFlagVec : 0u, {0u, 0u, 0u}});
+        starts.push_back(SegStart{(uint64_t)tiles.size(), numel[s], vec ? kSegFlagVec : 0u, (uint32_t)jobs.size(), {0u, 0u}});
+        const uint64_t first_tile = tiles.size();
         for (uint64_t off = 0; off < numel[s]; off += kSegTile) tiles.push_back(SegTile{s, vec ? kSegFlagVec : 0u, off});
+        for (uint64_t ft = first_tile; ft < tiles.size(); ft += kFoldJobTiles)
+            jobs.push_back(FoldJob{ft, (uint32_t)std::min<uint64_t>(kFoldJobTiles, tiles.size() - ft), s});
     }
     if (total != c->n) return A2SGD_ERR_ARG;
     DeviceGuard guard(c->device);
@@ -924,9 +931,12 @@ extern "C" int a2sgd_segments_create(a2sgd_ctx *c, uint32_t S, const uint64_t *n
     ok = ok && cudaMalloc(&sg->w, sizeof(float *) * w_count) == cudaSuccess;
     if (err) ok = ok && cudaMalloc(&sg->err, sizeof(float *) * (size_t)P * S) == cudaSuccess;
     ok = ok && cudaMemcpy(sg->tiles, tiles.data(), sizeof(SegTile) * tiles.size(), cudaMemcpyHostToDevice) == cudaSuccess;
-    starts.push_back(SegStart{(uint64_t)tiles.size(), 0, 0u, {0u, 0u, 0u}}); // end marker
+    starts.push_back(SegStart{(uint64_t)tiles.size(), 0, 0u, (uint32_t)jobs.size(), {0u, 0u}}); // end marker
+    sg->n_jobs = (uint32_t)jobs.size();
     ok = ok && cudaMalloc(&sg->starts, sizeof(SegStart) * starts.size()) == cudaSuccess;
     ok = ok && cudaMemcpy(sg->starts, starts.data(), sizeof(SegStart) * starts.size(), cudaMemcpyHostToDevice) == cudaSuccess;
+    ok = ok && cudaMalloc(&sg->fold_jobs, sizeof(FoldJob) * jobs.size()) == cudaSuccess;
+    ok = ok && cudaMemcpy(sg->fold_jobs, jobs.data(), sizeof(FoldJob) * jobs.size(), cudaMemcpyHostToDevice) == cudaSuccess;
     ok = ok && cudaMemcpy(sg->numel, numel, sizeof(uint64_t) * S, cudaMemcpyHostToDevice) == cudaSuccess;
     ok = ok && cudaMemcpy(sg->grad, grad, sizeof(float *) * (size_t)P * S, cudaMemcpyHostToDevice) == cudaSuccess;
     ok = ok && cudaMemcpy(sg->w, w, sizeof(float *) * w_count, cudaMemcpyHostToDevice) == cudaSuccess;
@@ -946,6 +956,8 @@ extern "C" int a2sgd_segments_destroy(a2sgd_segments *sg)
     DeviceGuard guard(sg->ctx->device);
     cudaFree(sg->tiles);
     cudaFree(sg->starts);
+    cudaFree(sg->fold_jobs);
+    cudaFree(sg->job_partials);
     cudaFree(sg->tile_partials);
     cudaFree(sg->seg_local_means);
     cudaFree(sg->seg_counts);
@@ -965,7 +977,10 @@ static SegTables seg_tables(const a2sgd_segments *sg, const float *lr_per_segmen
     t.tiles = sg->tiles;
     t.starts = sg->S <= kSegScanMax ? sg->starts : nullptr; // beyond that the decode kernel reads the tile table
     t.all_starts = sg->starts;
+    t.fold_jobs = sg->fold_jobs;
+    t.n_jobs = sg->n_jobs;
     t.tile_partials = sg->tile_partials;
+    t.job_partials = sg->job_partials;
     t.seg_local_means = sg->seg_local_means;
     t.seg_counts = sg->seg_counts;
     t.seg_global_means = sg->seg_global_means;
@@ -1043,12 +1058,15 @@ static int ensure_per_tensor_scratch(a2sgd_ctx *c, a2sgd_segments *sg)
     const size_t P = c->P, S = sg->S;
     bool ok = true;
     ok = ok && cudaMalloc(&sg->tile_partials, sizeof(Partial) * P * sg->n_tiles) == cudaSuccess;
+    ok = ok && cudaMalloc(&sg->job_partials, sizeof(Partial) * P * sg->n_jobs) == cudaSuccess;
     ok = ok && cudaMalloc(&sg->seg_local_means, sizeof(float) * 2 * P * S) == cudaSuccess;
     ok = ok && cudaMalloc(&sg->seg_counts, sizeof(unsigned long long) * P * S) == cudaSuccess;
     ok = ok && cudaMalloc(&sg->seg_global_means, sizeof(float) * 2 * S) == cudaSuccess;
     if (!ok) {
         (void)cudaGetLastError();
         cudaFree(sg->tile_partials);
+        cudaFree(sg->job_partials);
+        sg->job_partials = nullptr;
         cudaFree(sg->seg_local_means);
         cudaFree(sg->seg_counts);
         cudaFree(sg->seg_global_means);
@@ -1080,6 +1098,8 @@ extern "C" int a2sgd_step_segments_per_tensor(a2sgd_ctx *c, a2sgd_segments *sg, 
         SegTables t = seg_tables(sg, nullptr);
         uint32_t P = c->P;
         int *status = c->status;
+        void *params1[] = {&t};
+        A2_CUDA(launch_pdl(c->k->fold_jobs, dim3(sg->n_jobs, c->P), params1, s));
         void *params[] = {&t, &P, &status};
         A2_CUDA(launch_pdl(c->k->fold_segments, dim3(sg->S), params, s));
     }

@@ -21,5 +21,6 @@ struct a2sgd_kernel_table {
     const void *global_average;           // (const float *local_means, uint32_t P, float *out, float *ctx_copy)
     const void *global_average_from_sums; // (const double *sums, uint32_t workers, float *out, float *ctx_copy)
     const void *materialize_err;          // (float *v, int64_t stride, uint64_t n, const float *means)
+    const void *fold_jobs;                // (SegTables)
     const void *fold_segments;            // (SegTables, uint32_t P, int *status)
 };

@@ -32,7 +32,18 @@ struct __align__(16) SegStart {
     uint64_t first_tile;
     uint64_t numel;
     uint32_t flags;
-    uint32_t pad[3];
+    uint32_t first_job; // per-tensor-means variant: this tensor's fold jobs are [first_job, next entry's first_job)
+    uint32_t pad[2];
+};
+
+// Per-tensor-means variant: the per-tile partial sums of a tensor are added in two levels so that a
+// tensor of tens of thousands of tiles is not folded by a single CTA.  A job is a run of at most
+// kFoldJobTiles consecutive tiles of one tensor.
+constexpr uint32_t kFoldJobTiles = 1024;
+struct __align__(16) FoldJob {
+    uint64_t first_tile;
+    uint32_t count;
+    uint32_t seg;
 };
 constexpr uint32_t kSegScanMax = 4096; // tensors up to which the decode kernel scans SegStart (else: tile table)
 
@@ -49,7 +60,10 @@ struct SegTables {
     const float *lr_per_segment; // [S] device, or nullptr: one learning rate for the whole model
     // per-tensor-means variant only (plan-owned scratch)
     const SegStart *all_starts;        // [S + 1], always present
+    const FoldJob *fold_jobs;          // [n_jobs]
+    uint32_t n_jobs;
     Partial *tile_partials;            // [P][n_tiles]
+    Partial *job_partials;             // [P][n_jobs]
     float *seg_local_means;            // [S][P][2]
     unsigned long long *seg_counts;    // [S][P]
     float *seg_global_means;           // [S][2]
@@ -147,9 +161,35 @@ __global__ void __launch_bounds__(kBlock) k_encode_segments(EncodeArgs a, SegTab
     finish_worker(a, p, s_pos, s_neg, n_pos, sh_d, sh_n, &sh_flag);
 }
 
-// Per-tensor-means variant, between K1 and K3: block s adds the tile slots of tensor s in tile
-// order (thread t takes slots t, t + 256, ...; fixed tree above), one worker after the other, writes
-// that tensor's local means and counts, and averages them over the workers in worker order
+// Per-tensor-means variant, between K1 and K3, first level: block (j, p) adds the tile slots of job j
+// of worker p in tile order (thread t takes slots t, t + 256, ...; fixed tree above).  grid = (jobs, P).
+static __global__ void __launch_bounds__(kBlock) k_fold_jobs(SegTables t)
+{
+    pdl_wait_prior_grid();
+    pdl_release_next_grid();
+    __shared__ double sh_d[2][kWarps];
+    __shared__ unsigned long long sh_n[kWarps];
+    const FoldJob job = t.fold_jobs[blockIdx.x];
+    const uint32_t p = blockIdx.y;
+    const Partial *slot = t.tile_partials + (uint64_t)p * t.n_tiles + job.first_tile;
+    double s_pos = 0.0, s_neg = 0.0;
+    unsigned long long n_pos = 0;
+    for (uint32_t i = threadIdx.x; i < job.count; i += kBlock) {
+        s_pos += __ldcg(&slot[i].s_pos);
+        s_neg += __ldcg(&slot[i].s_neg);
+        n_pos += __ldcg(&slot[i].n_pos);
+    }
+    block_reduce(s_pos, s_neg, n_pos, sh_d, sh_n);
+    if (threadIdx.x == 0) {
+        Partial &out = t.job_partials[(uint64_t)p * t.n_jobs + blockIdx.x];
+        out.s_pos = s_pos;
+        out.s_neg = s_neg;
+        out.n_pos = n_pos;
+    }
+}
+
+// Second level: block s adds the job sums of tensor s in job order, one worker after the other,
+// writes that tensor's local means and counts, and averages them over the workers in worker order
 // (Algorithm 1 line 5, once per tensor).  grid = S.
 static __global__ void __launch_bounds__(kBlock) k_fold_segments(SegTables t, uint32_t P, int *status)
 {
@@ -158,14 +198,14 @@ static __global__ void __launch_bounds__(kBlock) k_fold_segments(SegTables t, ui
     __shared__ double sh_d[2][kWarps];
     __shared__ unsigned long long sh_n[kWarps];
     const uint32_t sg = blockIdx.x;
-    const uint64_t first = t.all_starts[sg].first_tile, last = t.all_starts[sg + 1].first_tile;
+    const uint32_t first = t.all_starts[sg].first_job, last = t.all_starts[sg + 1].first_job;
     const uint64_t numel = t.all_starts[sg].numel;
     double g_pos = 0.0, g_neg = 0.0; // thread 0: sums of the workers' means
     for (uint32_t p = 0; p < P; ++p) {
-        const Partial *slot = t.tile_partials + (uint64_t)p * t.n_tiles;
+        const Partial *slot = t.job_partials + (uint64_t)p * t.n_jobs;
         double s_pos = 0.0, s_neg = 0.0;
         unsigned long long n_pos = 0;
-        for (uint64_t i = first + threadIdx.x; i < last; i += kBlock) {
+        for (uint32_t i = first + threadIdx.x; i < last; i += kBlock) {
             s_pos += __ldcg(&slot[i].s_pos);
             s_neg += __ldcg(&slot[i].s_neg);
             n_pos += __ldcg(&slot[i].n_pos);

@@ -238,6 +238,7 @@ inline a2sgd_kernel_table kernel_table()
     t.global_average = (const void *)k_global_average;
     t.global_average_from_sums = (const void *)k_global_average_from_sums;
     t.materialize_err = (const void *)k_materialize_err;
+    t.fold_jobs = (const void *)k_fold_jobs;
     t.fold_segments = (const void *)k_fold_segments;
     return t;
 }
