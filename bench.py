@@ -456,6 +456,24 @@ def time_workload(wl, steps, warmup, dev, *, with_roofline=True, with_next_rows=
             torch.cuda.empty_cache()
 
     if with_e2e:
+        # every rank of the node holds its own host copy of the step's gradients: leave the leg out
+        # (and say so) rather than exhaust host memory when N ranks x P*n*4 bytes do not fit
+        try:
+            import psutil
+            host_free = psutil.virtual_memory().available
+        except Exception:
+            host_free = None
+        ranks_here = int(os.environ.get("LOCAL_WORLD_SIZE", "1"))
+        fits = not (host_free is not None and 1.25 * ranks_here * P * n * 4 > host_free)
+        if dist is not None:   # one decision for all ranks: the leg contains collectives
+            flag = torch.tensor([1.0 if fits else 0.0], device=dev, dtype=torch.float64)
+            dist.all_reduce(flag, op=dist.ReduceOp.MIN)
+            fits = bool(flag.item() > 0.5)
+        if not fits:
+            res["e2e_skipped"] = (f"{ranks_here} rank(s) x {P * n * 4 / 1e9:.1f} GB of host gradients do not fit in "
+                                  f"{(host_free or 0) / 1e9:.0f} GB of free host memory")
+            with_e2e = False
+    if with_e2e:
         pinned = True
         try:
             g_host = torch.empty((P, n), pin_memory=True)
@@ -827,11 +845,14 @@ def main():
         "config": config,
         "gpu_launches": res["launches"],
         "clocks": clocks,
-        "e2e": {"value": n_gpus * wl.n / (res["e2e_ms_per_step"] * 1e-3), "unit": UNIT,
-                "h2d_bytes_per_step": res["h2d_bytes"], "d2h_bytes_per_step": res["d2h_bytes"],
-                "ms_per_step": res["e2e_ms_per_step"], "ms_spread": res["e2e_ms_spread"], "steps": res["e2e_steps"],
-                "host_memory": "pinned" if res["e2e_pinned"] else "pageable (pinned allocation failed)",
-                "api": "a2sgd_step_host (pinned host gradients in, 2P+2 means out)"},
+        "e2e": ({"value": n_gpus * wl.n / (res["e2e_ms_per_step"] * 1e-3), "unit": UNIT,
+                 "h2d_bytes_per_step": res["h2d_bytes"], "d2h_bytes_per_step": res["d2h_bytes"],
+                 "ms_per_step": res["e2e_ms_per_step"], "ms_spread": res["e2e_ms_spread"], "steps": res["e2e_steps"],
+                 "host_memory": "pinned" if res["e2e_pinned"] else "pageable (pinned allocation failed)",
+                 "api": "a2sgd_step_host (pinned host gradients in, 2P+2 means out)"}
+                if "e2e_ms_per_step" in res else
+                {"value": None, "unit": UNIT, "h2d_bytes_per_step": wl.P * wl.n * 4, "d2h_bytes_per_step": (2 * wl.P + 2) * 4,
+                 "skipped": res.get("e2e_skipped", "not run")}),
         "roofline": dict(roofs["decode"], peak_source=peak_src,
                          traffic=traffic_per_el * wl.n if traffic_per_el else None,
                          traffic_source="ncu dram__bytes read+write per model element of a smaller capture of the "
