@@ -117,3 +117,39 @@ def test_the_check_fires_on_shrunk_extents_and_skips_the_access(P, n, stride):
     assert status == B.OK
     ctx.destroy()
     ctx2.destroy()
+
+
+@pytest.mark.parametrize("name", ["c4_vgg16", "c5_gpt2_xl"])
+def test_checked_kernels_at_full_benchmark_size(name):
+    """The 64-bit index arithmetic at the largest sizes (c5: 6.2 G worker-elements, byte offsets
+    beyond 2^34): the checked kernels latch nothing and produce the production kernels' bits
+    (compared through exact integer checksums of the bit patterns)."""
+    from paper_2006_07405_b200 import workloads as W
+    wl = W.get_workload(name)
+    n, P = wl.n, wl.P
+    free_dev, _ = torch.cuda.mem_get_info()
+    if (2 * P + 1) * n * 4 * 1.05 + (2 << 30) > free_dev:
+        pytest.skip("not enough device memory")
+    g = B.padded_rows(P, n, "cuda")
+    e = B.padded_rows(P, n, "cuda")
+    w = torch.empty(n, device="cuda")
+    W.fill_gradients(wl, 0, g)
+
+    def checksums():
+        parts = [w.view(torch.int32).sum(dtype=torch.int64)] + [e[p].view(torch.int32).sum(dtype=torch.int64)
+                                                              for p in range(P)]
+        return [int(x.item()) for x in parts]
+
+    sums = []
+    for flags in (EF, EF | B.DEBUG_CHECKS):
+        W.init_weights(wl, w)
+        gen = torch.Generator(device="cuda").manual_seed(123)
+        for p in range(P):
+            e[p].normal_(0.0, 1e-4, generator=gen)
+        ctx = B.a2sgd_create(n, P, 0, flags)
+        B.a2sgd_step(ctx, w, g, e, wl.lr)
+        lm, gm, cnt, status = B.a2sgd_read_stats(ctx)
+        assert status == B.OK, B.status_string(status)
+        sums.append((checksums(), lm.tobytes(), gm.tobytes(), cnt.tobytes()))
+        ctx.destroy()
+    assert sums[0] == sums[1]
