@@ -116,8 +116,9 @@ enum a2sgd_flags {
                                          faults.  For segment lists the check is on tile and tensor indices
                                          instead of addresses.  The extents live in one descriptor per device, so
                                          calls of a checking context must not overlap other calls of the library
-                                         on the same device (different streams or threads).  Several times
-                                         slower; off by default. */
+                                         on the same device (different streams or threads), and they cannot be
+                                         captured into a CUDA graph (A2SGD_ERR_CUDA during capture).  Several
+                                         times slower; off by default. */
     A2SGD_TEST_SHRINK_EXTENTS = 1 << 11, /* test hook for A2SGD_DEBUG_CHECKS: the extents recorded for a call are
                                             one element per row short, so the checked kernels skip every access
                                             that touches a row's last element and latch A2SGD_ERR_BOUNDS — the

@@ -428,6 +428,13 @@ struct DebugScope {
     bool arm(int mode)
     {
         if (!(c->flags & A2SGD_DEBUG_CHECKS)) return true;
+        // the descriptor is copied from this (stack) object: a captured copy would read it again at
+        // every replay, long after it is gone — checking contexts are refused during stream capture
+        cudaStreamCaptureStatus capturing = cudaStreamCaptureStatusNone;
+        if (cudaStreamIsCapturing(s, &capturing) != cudaSuccess || capturing != cudaStreamCaptureStatusNone) {
+            (void)cudaGetLastError();
+            return false;
+        }
         d.on = mode;
         d.status = c->status;
         armed = a2sgd_checked_arm(&d, sizeof(d), s) == cudaSuccess;

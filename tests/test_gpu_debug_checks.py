@@ -153,3 +153,25 @@ def test_checked_kernels_at_full_benchmark_size(name):
         sums.append((checksums(), lm.tobytes(), gm.tobytes(), cnt.tobytes()))
         ctx.destroy()
     assert sums[0] == sums[1]
+
+
+def test_checking_context_is_refused_during_stream_capture():
+    """The extents of a checked call are handed to the device from a short-lived host object, so a
+    captured call would replay a dangling copy: the library refuses instead."""
+    P, n = 2, 4096
+    g, e, w = _inputs(3, P, n, n, False)
+    ctx = B.a2sgd_create(n, P, 0, EF | B.DEBUG_CHECKS)
+    B.a2sgd_step(ctx, w, g, e, 0.1)                          # outside capture: fine
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            with pytest.raises(B.A2SGDError) as ei:
+                B.a2sgd_step(ctx, w, g, e, 0.1, stream=side)
+            w.add_(0.0)                                      # something harmless to capture
+    assert ei.value.status == B.ERR_CUDA
+    torch.cuda.current_stream().wait_stream(side)
+    *_, status = B.a2sgd_read_stats(ctx)
+    assert status == B.OK
+    ctx.destroy()
