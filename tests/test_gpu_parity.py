@@ -715,3 +715,37 @@ def test_f16_gradient_step_matches_oracle_on_widened_gradients(mode, replicated,
     assert_means(gm, gm_ref)
     assert_state(w.cpu().numpy(), wh, e.cpu().numpy(), eh, gm_ref, f"f16 P={P} n={n}")
     ctx.destroy()
+
+
+def test_average_from_allreduced_sums_matches_oracle():
+    """Algorithm 1 line 5 in its all-reduce form: the collective delivers fp64 sums of the pairs,
+    the library divides.  Reference: the oracle's global average of the same pairs."""
+    rng = np.random.default_rng(4)
+    for W_ in (1, 2, 3, 8, 64):
+        lm = (rng.random((W_, 2)) * 1e-3).astype(np.float32)
+        sums = torch.from_numpy(lm.astype(np.float64).sum(0)).cuda()      # what an all-reduce(SUM) returns
+        ctx = B.a2sgd_create(1000, 1, 0, EF)
+        gm = torch.zeros(2, device="cuda")
+        B.a2sgd_global_average_from_sums(ctx, sums, W_, gm)
+        assert_means(gm.cpu().numpy(), oracle.global_average(lm))
+        ctx.destroy()
+
+
+def test_dense_sync_on_an_allreduced_sum_matches_oracle():
+    """Algorithm 1 lines 9-10 with one worker per GPU: the all-reduced SUM of the gradients goes in,
+    the library divides by the worker count."""
+    rng = np.random.default_rng(6)
+    n, W_ = 100_003, 4
+    g = (rng.standard_normal((W_, n)) * 1e-3).astype(np.float32)
+    w0 = (rng.standard_normal(n) * 0.02).astype(np.float32)
+    g_sum = torch.from_numpy(g).cuda().sum(0)                               # fp32 sum, as NCCL would form it
+    w = torch.from_numpy(w0).cuda()
+    ctx = B.a2sgd_create(n, 1, 0, EF)
+    B.a2sgd_dense_sync_reduced(ctx, w, g_sum, W_, 0.1)
+    w_ref = w0.copy()
+    oracle.dense_sync(w_ref, g, 0.1)
+    assert_state(w.cpu().numpy(), w_ref, None, None, None, "dense sync on a reduced sum")
+    with pytest.raises(B.A2SGDError):                                       # contexts of one worker only
+        ctx4 = B.a2sgd_create(n, 4, 0, EF)
+        B.a2sgd_dense_sync_reduced(ctx4, w, g_sum, W_, 0.1)
+    ctx.destroy()
