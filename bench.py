@@ -434,6 +434,9 @@ def time_workload(wl, steps, warmup, dev, *, with_roofline=True, with_next_rows=
             B.a2sgd_materialize_err(dctx, e)
             torch.cuda.synchronize(dev)
             dctx.destroy()
+        actx = B.a2sgd_create(n, P, dev.index, B.MODE_ALG1)
+        res["step_alg1_ms"] = timed(lambda: B.a2sgd_step(actx, w, g, None, wl.lr))
+        actx.destroy()
         mom = torch.zeros(n, device=dev)
         res["step_momentum_ms"] = timed(lambda: B.a2sgd_step_momentum(ctx, w, mom, g, e, wl.lr, 0.9, 1e-4))
         del mom
@@ -587,6 +590,12 @@ def next_rows_of(wl, res, peak_gbs) -> dict:
             "model_params_per_s": wl.n / (res["step_deferred_ms"] * 1e-3),
             "bytes_per_model_element": 12 * wl.P + 8 + wl.P / 4,
             "speedup_vs_canonical_step": res["ms_per_step"] / res["step_deferred_ms"]}
+    if "step_alg1_ms" in res:
+        bts = (8 * wl.P + 8) * wl.n
+        rows["step in ALG1 mode (Algorithm 1 as printed: same-iteration add-back, eps not stored)"] = {
+            "ms": res["step_alg1_ms"], "GBps": bts / (res["step_alg1_ms"] * 1e-3) / 1e9,
+            "frac_of_8TBps": bts / (res["step_alg1_ms"] * 1e-3) / 1e9 / NOMINAL_HBM_GBS,
+            "model_params_per_s": wl.n / (res["step_alg1_ms"] * 1e-3), "bytes_per_model_element": 8 * wl.P + 8}
     if "step_momentum_ms" in res:
         bts = (20 * wl.P + 16) * wl.n
         rows["step with momentum and weight decay (a2sgd_step_momentum)"] = {
