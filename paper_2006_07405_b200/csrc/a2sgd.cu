@@ -29,12 +29,16 @@ cudaError_t a2sgd_checked_arm(const void *descriptor, size_t bytes, cudaStream_t
 //    SMs do not stream at equal speed (two dies, shared channels), so the slowest share set the
 //    time.  Letting the hardware CTA scheduler hand out small CTAs reaches 6.9-7.0 TB/s.
 //  * encode: per-CTA partial sums must stay few and their order fixed, so the grid stays
-//    proportional to the resident-CTA count: 16 CTAs per resident slot (1 -> 2 -> 4 -> 16 measured
-//    7.18 -> 7.27 -> 7.33 -> 7.36 TB/s on c5 and 7.02 -> 7.13 -> 7.18 -> 7.24 on c4; the fold of
-//    the 18944 / P partials per worker by the last CTA stays negligible).  The deferred-residual
-//    encode also writes v, a read/write mix, and gains the same way (c2: 626 us per step at 1,
-//    583 at 16 and 32, 599 at 64).
+//    proportional to the resident-CTA count: 16 CTAs per resident slot, 32 from half a billion
+//    worker-elements up (c5, us per launch at 2 / 4 / 8 / 16 / 32 / 64: 6853 / 6796 / 6772 / 6773 /
+//    6685 / 6668; c4: 620 / 617 / 617 / 612 / 606 / 610; c2: 300 / 303 / 305 / 300 / 304 / 329 —
+//    smaller CTAs shorten the tail of the grid, more of them lengthen the last CTA's fold of the
+//    partial sums, which the small configurations feel first).  The deferred-residual encode also
+//    writes v, a read/write mix, and gains the same way (c2: 626 us per step at 1, 583 at 16 and 32,
+//    599 at 64).
 constexpr int kWavesK1 = 16;
+constexpr int kWavesK1Large = 32;
+constexpr uint64_t kLargeWorkerElements = 1ull << 29;
 constexpr int kWavesK1Deferred = 16;
 constexpr int kWavesK3 = 1 << 20; // effectively: cover every vector with its own thread
 constexpr int kMaxVecWidth = 8;   // widest access the dispatcher picks: 256-bit
@@ -65,6 +69,11 @@ struct a2sgd_ctx {
     // resident CTAs per SM of every kernel instance used so far (occupancy API, cached)
     std::unordered_map<const void *, int> occ;
 };
+
+inline int encode_waves(const a2sgd_ctx *c)
+{
+    return c->n * (uint64_t)c->P >= kLargeWorkerElements ? kWavesK1Large : kWavesK1;
+}
 
 struct a2sgd_segments {
     a2sgd_ctx *ctx = nullptr;
@@ -249,7 +258,7 @@ int launch_encode(a2sgd_ctx *c, const float *grad, int64_t gs, const float *err,
     EncodeArgs a = make_encode_args(c, grad, gs, err, es, local_means, pos_counts, pos_mask, global_means);
     const void *fn = c->k->encode(!c->alg1, pos_mask != nullptr, vw);
     const uint64_t items = vw ? (c->n + vw - 1) / vw : (c->n + kScalarU - 1) / kScalarU;
-    const dim3 grid(std::min(per_worker_grid(c, occupancy(c, fn), items, kWavesK1), c->g_alloc), c->P);
+    const dim3 grid(std::min(per_worker_grid(c, occupancy(c, fn), items, encode_waves(c)), c->g_alloc), c->P);
     void *params[] = {&a};
     A2_CUDA(launch_pdl(fn, grid, params, s));
     return A2SGD_OK;
@@ -502,7 +511,7 @@ extern "C" int a2sgd_create(a2sgd_ctx **out, uint64_t n, uint32_t P, int device,
         c->l2_bytes = (size_t)std::max(l2, 0);
     }
     // partials: room for a (G, P) grid that fills the device at the highest possible occupancy
-    const uint32_t max_slots = (uint32_t)c->sm_count * (2048 / kBlock) * std::max(kWavesK1, kWavesK1Deferred);
+    const uint32_t max_slots = (uint32_t)c->sm_count * (2048 / kBlock) * std::max(kWavesK1Large, kWavesK1Deferred);
     c->g_alloc = std::max<uint32_t>(1, max_slots / P);
     bool ok = true;
     ok = ok && cudaMalloc(&c->partials, sizeof(Partial) * (size_t)c->g_alloc * P) == cudaSuccess;
@@ -789,7 +798,7 @@ static int step_lowp(a2sgd_ctx *c, float *w, int64_t w_stride, const uint16_t *g
                                         c->global_means);
         const void *fn = c->k->encode_lowp(gt, ef, vw_enc);
         const uint64_t items = vw_enc ? (c->n + 7) / 8 : (c->n + kScalarU - 1) / kScalarU;
-        const dim3 grid(std::min(per_worker_grid(c, occupancy(c, fn), items, kWavesK1), c->g_alloc), c->P);
+        const dim3 grid(std::min(per_worker_grid(c, occupancy(c, fn), items, encode_waves(c)), c->g_alloc), c->P);
         void *params[] = {&a};
         A2_CUDA(launch_pdl(fn, grid, params, s));
     }
@@ -1009,7 +1018,7 @@ static int launch_encode_segments(a2sgd_ctx *c, a2sgd_segments *sg, float *local
     SegTables t = seg_tables(sg, nullptr);
     EncodeArgs a = make_encode_args(c, nullptr, 0, nullptr, 0, local_means, pos_counts, nullptr, global_means);
     const void *fn = c->k->encode_segments(!c->alg1, per_tensor);
-    const uint64_t slots = (uint64_t)c->sm_count * occupancy(c, fn) * kWavesK1;
+    const uint64_t slots = (uint64_t)c->sm_count * occupancy(c, fn) * encode_waves(c);
     uint64_t G = std::max<uint64_t>(1, slots / c->P);
     G = std::min<uint64_t>(std::min<uint64_t>(G, sg->n_tiles), c->g_alloc);
     void *params[] = {&a, &t};
@@ -1228,7 +1237,7 @@ extern "C" int a2sgd_launch_info(a2sgd_ctx *c, int64_t w_stride, uint32_t out[5]
     const bool shared = w_stride == 0 || c->P == 1;
     const int vw = kMaxVecWidth >= 8 ? 8 : 4;
     const uint64_t items = (c->n + vw - 1) / vw;
-    out[0] = std::min(per_worker_grid(c, occupancy(c, c->k->encode(ef, false, vw)), items, kWavesK1),
+    out[0] = std::min(per_worker_grid(c, occupancy(c, c->k->encode(ef, false, vw)), items, encode_waves(c)),
                       c->g_alloc) * c->P;
     out[1] = shared ? flat_grid(c, occupancy(c, c->k->decode_shared(ef, true, c->P, vw, false)), items, kWavesK3)
                     : per_worker_grid(c, occupancy(c, c->k->decode_repl(ef, true, vw, false)), items, kWavesK3) * c->P;
