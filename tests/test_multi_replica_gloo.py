@@ -144,3 +144,30 @@ def test_exchange_leg_protocol_world_size_2(tmp_path):
     for r, (p, out) in enumerate(zip(procs, outs)):
         assert p.returncode == 0, out
         assert f"rank {r} ok" in out
+
+
+def test_bench_line_helpers():
+    """The pure helpers behind the JSON line: spread of per-step times, per-kernel roofline records
+    (algorithmic bytes / launch time against the peak) and the rows beyond the plain step."""
+    sys.path.insert(0, ROOT)
+    import bench
+    from paper_2006_07405_b200 import workloads as W
+    s = bench.spread([3.0, 1.0, 2.0, 10.0])
+    assert s == {"median": 2.5, "min": 1.0, "max": 10.0, "n": 4}
+    assert bench.spread([]) == {"n": 0}
+    wl = W.get_workload("c4_vgg16")
+    res = {"encode_ms": 0.6, "decode_ms": 1.1, "encode_ms_spread": s, "decode_ms_spread": s}
+    roofs = bench.kernel_rooflines(wl, res, 6529.7)
+    dec = roofs["decode"]
+    assert dec["bound"] == "hbm" and dec["unit"] == "GB/s" and dec["peak"] == 6529.7
+    assert dec["algorithmic_bytes"] == (12 * wl.P + 8) * wl.n
+    assert abs(dec["achieved"] - dec["algorithmic_bytes"] / 1.1e-3 / 1e9) < 1e-6
+    assert abs(dec["frac"] - dec["achieved"] / 6529.7) < 1e-12
+    assert roofs["encode"]["algorithmic_bytes"] == 8 * wl.P * wl.n
+    rows = bench.next_rows_of(wl, {"ms_per_step": 1.7, "dense_sync_ms": 0.46, "step_momentum_ms": 1.9,
+                                   "step_alg1_ms": 0.8, "step_bf16_ms": 1.45}, 6529.7)
+    assert len(rows) == 4
+    mom = rows["step with momentum and weight decay (a2sgd_step_momentum)"]
+    assert mom["bytes_per_model_element"] == 20 * wl.P + 16
+    assert set(bench.host_description()) == {"nproc", "usable_cores", "cpu_model"}
+    assert bench.NCU_DECODE_TRAFFIC_PER_ELEMENT[4] < 12 * 4 + 8 < bench.NCU_DECODE_TRAFFIC_PER_ELEMENT[8]
