@@ -87,7 +87,8 @@ enum a2sgd_flags {
     A2SGD_FORCE_COOPERATIVE = 1 << 5, /* a2sgd_step takes the single-launch path whenever (n, P) fits it — v in
                                          registers, or g, e, w within 70 % of L2 — and returns
                                          A2SGD_ERR_TOO_LARGE otherwise.  Without this flag the single launch is
-                                         used only where it measured faster: one worker, v in registers. */
+                                         used only where it measured faster: v in registers with one CTA per SM
+                                         (n*P up to about 1.2 M elements), or one worker with v in registers. */
     A2SGD_DEFERRED_RESIDUAL = 1 << 7, /* EF mode only, opt-in: between steps the caller's error buffer holds the
                                          compensated vector v of the last step instead of the residual
                                          e = v - g_hat(v); the subtraction is done one step later, with the

@@ -312,28 +312,32 @@ int launch_decode(a2sgd_ctx *c, float *w, int64_t ws, const float *grad, int64_t
 // per thread.  L2-resident form: g, e and w together within 70 % of the L2 capacity.
 // Returns the kernel and its grid, or nullptr when (n, P, alignment) does not qualify.
 //
-// Which sizes take it by default is decided by measurement (B200, CUDA graphs of 20 steps, us per
-// step, single launch vs two launches): P = 1: 1 M 9.6 vs 10.6, 2 M 11.2 vs 14.5 (register form);
-// 4 M 18.4 vs 18.1 (L2 form).  P = 2, 0.5 M: 11.1 vs 10.1.  P = 4: 0.25 M 11.0 vs 10.6, 0.5 M 13.6
-// vs 12.5, 1 M (L2 form) 17.1 vs 15.8.  The two-launch path hands its decode work to the hardware
-// CTA scheduler one vector per thread, which balances the SMs better than the equal static shares
-// a co-resident grid must use, and that outweighs the saved launch except for a single worker with
-// v in registers.  So: automatic only for P = 1 in the register form; everything else that fits is
-// available through A2SGD_FORCE_COOPERATIVE.
+// Which sizes take it by default is decided by measurement (B200, CUDA graphs of 50 steps, us per
+// step, single launch vs two launches).  With one CTA per SM (v of all workers fits the registers of
+// 148 CTAs: n * P <= 1.2 M elements) the single launch wins for every worker count: P = 1, 1 M: 8.7 vs
+// 10.8; P = 2, 0.6 M: 9.2 vs 10.4; P = 4, 0.3 M: 9.9 vs 10.9; P = 8, 0.15 M: 9.9 vs 12.4.  Needing
+// two or three CTAs per SM it still wins for one worker (1.5 M: 10.5 vs 10.8; 2 M: 11.5 vs 13.9) but
+// not in general for several (P = 4, 0.5 M: 14.2 vs 12.4; P = 2, 0.8 M: 12.3 vs 10.9): the arrivals
+// at the grid barrier double or triple, and the two-launch path hands its decode work to the
+// hardware CTA scheduler, which balances the SMs better than equal static shares.  So: automatic
+// for the register form when one CTA per SM is enough or P = 1; everything else that fits
+// (including the L2-resident form: 1 M x 4: 17.1 vs 15.8) is available through A2SGD_FORCE_COOPERATIVE.
 const void *coop_plan(a2sgd_ctx *c, bool store, bool shared, int vw, uint32_t *grid_out)
 {
     if (!c->coop_supported || vw < 4) return nullptr;
     const bool forced = (c->flags & A2SGD_FORCE_COOPERATIVE) != 0;
-    if (!forced && c->P != 1) return nullptr;
     const void *fn = c->k->coop(!c->alg1, store, shared, c->P);
     if (!fn) return nullptr;
     const uint64_t n4 = (c->n + 3) / 4;
     const uint64_t need = std::max<uint64_t>(1, (n4 + kBlock - 1) / kBlock);
-    {
-        const uint64_t resident = (uint64_t)c->sm_count * occupancy(c, fn);
+    // The smallest co-resident grid whose registers hold v: one CTA per SM where that is enough (half
+    // the arrivals at the grid barrier: c1 9.6 -> 8.7 us per step), full occupancy otherwise.
+    for (const int ctas_per_sm : {1, occupancy(c, fn)}) {
+        const uint64_t resident = (uint64_t)c->sm_count * ctas_per_sm;
         const uint64_t per_thread = kCoopVecPerThread / c->P;
         const uint64_t grid = std::min<uint64_t>(resident, need);
         if (n4 <= resident * kBlock * per_thread && grid <= c->g_alloc) {
+            if (!forced && ctas_per_sm != 1 && c->P != 1) return nullptr; // measured slower than two launches
             *grid_out = (uint32_t)grid;
             return fn;
         }
