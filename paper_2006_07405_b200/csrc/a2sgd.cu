@@ -363,7 +363,22 @@ int launch_coop(a2sgd_ctx *c, const void *fn, uint32_t grid, float *w, int64_t w
     a.expected = never_opens ? grid + 1 : grid;
     a.spin_limit = never_opens ? (1u << 12) : (1u << 24); // x 40 ns sleep: ~0.2 ms / ~1 s
     void *params[] = {&a};
-    A2_CUDA(cudaLaunchCooperativeKernel(fn, dim3(grid), dim3(kBlock), params, 0, s));
+    // cooperative (all CTAs co-resident: the grid barrier needs it) and, like the other kernels,
+    // with programmatic stream serialisation: the CTAs of the next step may become resident while
+    // this grid drains; they wait for it before their first memory access, ahead of the barrier
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(kBlock);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeCooperative;
+    attr[0].val.cooperative = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 2;
+    A2_CUDA(cudaLaunchKernelExC(&cfg, fn, params));
     return A2SGD_OK;
 }
 

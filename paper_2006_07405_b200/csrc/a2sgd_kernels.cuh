@@ -1465,6 +1465,8 @@ __device__ __forceinline__ void coop_worker_consts(const EncodeArgs &ea, WorkerC
 template <bool EF, bool STORE, int PT, bool SHARED>
 __global__ void __launch_bounds__(kBlock) k_step_coop(CoopArgs a)
 {
+    pdl_wait_prior_grid();
+    pdl_release_next_grid();
     constexpr int K = kCoopVecPerThread / PT;
     __shared__ CoopShared<PT> sh;
 
@@ -1575,6 +1577,8 @@ __global__ void __launch_bounds__(kBlock) k_step_coop(CoopArgs a)
 template <bool EF, bool STORE, int PT, bool SHARED>
 __global__ void __launch_bounds__(kBlock) k_step_coop_l2(CoopArgs a)
 {
+    pdl_wait_prior_grid();
+    pdl_release_next_grid();
     __shared__ CoopShared<PT> sh;
     const EncodeArgs &ea = a.enc;
     const DecodeArgs &da = a.dec;
