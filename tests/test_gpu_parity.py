@@ -749,3 +749,37 @@ def test_dense_sync_on_an_allreduced_sum_matches_oracle():
         ctx4 = B.a2sgd_create(n, 4, 0, EF)
         B.a2sgd_dense_sync_reduced(ctx4, w, g_sum, W_, 0.1)
     ctx.destroy()
+
+
+def test_pointer_check_flag_covers_the_other_entry_points():
+    """A2SGD_CHECK_POINTERS on the momentum, 16-bit-gradient, staged, reduced-sum and segment-list
+    calls: a host address comes back as A2SGD_ERR_ARG before anything is launched."""
+    import ctypes
+    n, P = 4096, 2
+    g = B.padded_rows(P, n, "cuda", 0.0)
+    e = B.padded_rows(P, n, "cuda", 0.0)
+    w = torch.zeros(n, device="cuda")
+    m = torch.zeros(n, device="cuda")
+    lm = torch.zeros((P, 2), device="cuda")
+    gm = torch.zeros(2, device="cuda")
+    host = np.zeros((P, n), np.float32)
+    hp = host.ctypes.data
+    ctx = B.a2sgd_create(n, P, 0, EF | B.CHECK_POINTERS)
+    h, lib, s = ctx.handle, B.lib(), g.stride(0)
+    assert lib.a2sgd_step_momentum(h, w.data_ptr(), 0, hp, 0, g.data_ptr(), s, e.data_ptr(), s, 0.1, 0.9, 0.0, None) == B.ERR_ARG
+    assert lib.a2sgd_step_bf16(h, w.data_ptr(), 0, hp, n, e.data_ptr(), s, 0.1, None) == B.ERR_ARG
+    assert lib.a2sgd_global_average(h, hp, gm.data_ptr(), None) == B.ERR_ARG
+    assert lib.a2sgd_global_average_from_sums(h, hp, 2, gm.data_ptr(), None) == B.ERR_ARG
+    assert lib.a2sgd_encode(h, g.data_ptr(), s, e.data_ptr(), s, hp, None, None, None) == B.ERR_ARG
+    assert lib.a2sgd_decode_update(h, w.data_ptr(), 0, g.data_ptr(), s, e.data_ptr(), s, lm.data_ptr(), hp, 0.1, None) == B.ERR_ARG
+    vp = ctypes.c_void_p
+    numel = (ctypes.c_uint64 * 1)(n)
+    g_tab = (vp * 2)(g[0].data_ptr(), hp)                     # worker 1's gradient tensor lives on the host
+    e_tab = (vp * 2)(e[0].data_ptr(), e[1].data_ptr())
+    w_tab = (vp * 1)(w.data_ptr())
+    out = vp()
+    assert lib.a2sgd_segments_create(h, 1, numel, g_tab, e_tab, w_tab, 0, ctypes.byref(out)) == B.ERR_ARG and not out
+    B.a2sgd_step_momentum(ctx, w, m, g, e, 0.1, 0.9, 0.0)     # device buffers pass
+    *_, status = B.a2sgd_read_stats(ctx)
+    assert status == B.OK
+    ctx.destroy()
